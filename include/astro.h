@@ -1,0 +1,143 @@
+/*
+ * astro.h -- C ABI of the rolling-KV chunk-attention library (sm_100a).
+ *
+ * One DiT layer's self-attention in the streaming scheme: the queries of a new
+ * chunk of latent frames attend to a restricted context (S permanently kept
+ * "sink" frames plus a sliding window of recent frames) and to the chunk itself.
+ *
+ * Conventions shared by every call
+ *   - Every data pointer is a DEVICE pointer to memory the caller allocated and
+ *     keeps alive; the library frees none of it.  The cache handle owns only
+ *     host-side metadata.  Query outputs (int*, int64_t*) are HOST pointers.
+ *   - Work is enqueued on the given CUDA stream (passed as void*, a cudaStream_t)
+ *     and the call returns without synchronising.  Calls on one cache must come
+ *     from one host thread; metadata changes take effect in call order.
+ *   - bf16 tensors Q, O, K_chunk, V_chunk, dO, dQ, dK_chunk, dV_chunk are
+ *     contiguous [batch, tokens, heads, head_dim].  LSE and delta are fp32
+ *     [batch, heads, tokens].  Data pointers must be 16-byte aligned.
+ *   - Functions return ASTRO_OK or an error code; they never throw or exit, and
+ *     on an error the cache metadata is unchanged and nothing was launched.
+ */
+#ifndef ASTRO_H_
+#define ASTRO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct astro_kvcache astro_kvcache_t; /* opaque, host side */
+
+typedef enum {
+  ASTRO_OK = 0,
+  ASTRO_ERR_NULL = 1,      /* a required pointer is null */
+  ASTRO_ERR_SHAPE = 2,     /* unsupported or inconsistent shape (head_dim not 64/128, batch mismatch, empty key set) */
+  ASTRO_ERR_ALIGN = 3,     /* a data pointer is not 16-byte aligned */
+  ASTRO_ERR_CAPACITY = 4,  /* append would hold more than S+L frames, or a buffer is too small */
+  ASTRO_ERR_UNDERFLOW = 5, /* evict asks for more window frames than are held */
+  ASTRO_ERR_ARCH = 6,      /* current device is not compute capability 10.x */
+  ASTRO_ERR_CUDA = 7,      /* a CUDA runtime/driver call failed */
+  ASTRO_ERR_TIMEOUT = 8    /* a bounded device-side wait ran out (see astro_last_device_status) */
+} astro_status_t;
+
+typedef struct {
+  int cache_batch;      /* B_c: samples with their own cache; 1 = one shared frozen prefix for a group */
+  int heads;            /* H */
+  int head_dim;         /* D: 64 or 128 */
+  int tokens_per_frame; /* T */
+  int sink_frames;      /* S >= 0 */
+  int window_frames;    /* L >= 1: slots of the sliding window */
+} astro_kvcache_desc_t;
+
+/* Bytes the caller must allocate for K (and the same again for V):
+ * B_c * H * (S+L) * T * D * 2.  Returns 0 for an invalid descriptor. */
+size_t astro_kvcache_storage_bytes(const astro_kvcache_desc_t* desc);
+
+/* Sec. 3.2, "Rolling KV Cache with Frame Sinks": bind caller-allocated device
+ * storage for the restricted context C_n (S sink frames + window of L frames),
+ * so that resident KV memory is constant however long the video grows.
+ * k_storage/v_storage: device, >= bytes_each each, 1024-byte aligned; the layout
+ * inside is private ([B_c, H, slot, T, D]).  The storage need not be initialised.
+ * The cache starts empty.  *out receives the handle. */
+astro_status_t astro_kvcache_create(const astro_kvcache_desc_t* desc, void* k_storage, void* v_storage,
+                                    size_t bytes_each, astro_kvcache_t** out);
+
+/* Frees the host-side handle only. */
+astro_status_t astro_kvcache_destroy(astro_kvcache_t* cache);
+
+/* Empties the cache (the next S appended frames become the new sink); storage is kept. */
+astro_status_t astro_kvcache_reset(astro_kvcache_t* cache);
+
+/* Sec. 3.3, "Streaming Long Tuning" (the forward pass accumulates the KV cache up
+ * to the target step) and Sec. 3.2: store K and V of n_frames new frames.
+ * k, v: device bf16 [B_c, n_frames*T, H, D].  The first S frames ever appended
+ * fill the sink; later ones take the next free window slot.  The copy is
+ * bit-exact.  There is no implicit eviction: ASTRO_ERR_CAPACITY if the cache
+ * would hold more than S+L frames. */
+astro_status_t astro_kvcache_append(astro_kvcache_t* cache, const void* k, const void* v, int n_frames,
+                                    void* stream);
+
+/* Sec. 3.2: the window keeps "the L most recent frames": drop the n_frames
+ * oldest window frames.  Sink frames are never dropped.  The window is a ring,
+ * so this advances an index and moves no bytes (the stream is unused today).
+ * ASTRO_ERR_UNDERFLOW if n_frames exceeds the window frames held. */
+astro_status_t astro_kvcache_evict(astro_kvcache_t* cache, int n_frames, void* stream);
+
+/* Host-side state: frames held in the sink, in the window, and frames appended
+ * since create/reset.  Any of the three HOST pointers may be null. */
+astro_status_t astro_kvcache_query(const astro_kvcache_t* cache, int* sink_held, int* window_held,
+                                   int64_t* frames_seen);
+
+/* Inspection aid: write the held frames in logical order (sink frames, then
+ * window oldest to newest) to k_out, v_out: device bf16 [B_c, held*T, H, D]. */
+astro_status_t astro_kvcache_export(const astro_kvcache_t* cache, void* k_out, void* v_out, void* stream);
+
+/* Sec. 3.2 (the model "attends exclusively to the KV cache of C_n" while it
+ * generates the next clip; G candidates decode against one shared prefix) --
+ * forward of chunk attention.  For every sample b, head h and chunk query i:
+ *   keys/values = every token held in the cache (of sample b, or of the single
+ *   shared cache when B_c = 1) followed by the n_kc chunk tokens;
+ *   s_ij = scale * q_i . k_j;  LSE_i = ln sum_j exp(s_ij);  o_i = sum_j exp(s_ij - LSE_i) v_j.
+ * q [batch, n_q, H, D], k_chunk/v_chunk [batch, n_kc, H, D] (may be null when
+ * n_kc = 0), o [batch, n_q, H, D] bf16, lse [batch, H, n_q] fp32 (may be null).
+ * cache may be null (no context).  n_q, n_kc are token counts and need not be
+ * multiples of T or of any tile.  ASTRO_ERR_SHAPE if there is no key at all, or
+ * batch differs from B_c and B_c != 1.  bf16 products, fp32 accumulation and softmax. */
+astro_status_t astro_chunk_attn_fwd(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
+                                    const void* v_chunk, int batch, int heads, int head_dim, int n_q,
+                                    int n_kc, float scale, void* o, float* lse, void* stream);
+
+/* Scratch bytes astro_chunk_attn_bwd needs (delta, fp32 [batch, H, n_q], rounded up). */
+size_t astro_chunk_attn_bwd_workspace_bytes(int batch, int heads, int n_q, int head_dim);
+
+/* Sec. 3.3, "Streaming Long Tuning": the KV cache of all preceding frames is
+ * detached; gradients flow through the active window only.  Given dO and the
+ * forward's O and LSE:
+ *   p_ij = exp(s_ij - LSE_i); dp_ij = dO_i . v_j; delta_i = dO_i . o_i;
+ *   ds_ij = p_ij (dp_ij - delta_i);
+ *   dq_i = scale * sum over ALL keys of ds_ij k_j;
+ *   dk_j = scale * sum_i ds_ij q_i and dv_j = sum_i p_ij dO_i for CHUNK keys only.
+ * dq [batch, n_q, H, D], dk_chunk/dv_chunk [batch, n_kc, H, D], all bf16 written
+ * from fp32 accumulators (dk_chunk/dv_chunk may be null when n_kc = 0).
+ * workspace: device scratch of at least astro_chunk_attn_bwd_workspace_bytes(). */
+astro_status_t astro_chunk_attn_bwd(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
+                                    const void* v_chunk, const void* o, const float* lse, const void* d_o,
+                                    int batch, int heads, int head_dim, int n_q, int n_kc, float scale,
+                                    void* dq, void* dk_chunk, void* dv_chunk, void* workspace,
+                                    size_t workspace_bytes, void* stream);
+
+/* Every device-side wait in the kernels is bounded; one that runs out records a
+ * code in a device status word instead of hanging.  This call synchronises the
+ * current device, reads and clears that word: ASTRO_OK, or ASTRO_ERR_TIMEOUT
+ * (then *detail, a HOST pointer that may be null, receives the raw word). */
+astro_status_t astro_last_device_status(uint32_t* detail);
+
+/* Static, never null. */
+const char* astro_status_string(astro_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASTRO_H_ */

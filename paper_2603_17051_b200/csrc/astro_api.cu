@@ -1,0 +1,445 @@
+// C ABI of the rolling-KV chunk-attention library: host-side cache metadata, argument checks,
+// tensor-map construction and kernel launches.  Declarations and semantics: include/astro.h.
+#include "astro.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstring>
+#include <mutex>
+#include <new>
+
+#include "attn_bwd.cuh"
+#include "attn_fwd.cuh"
+#include "kv_ring.cuh"
+
+using namespace astro;
+
+struct astro_kvcache {
+  astro_kvcache_desc_t d;
+  void* k;
+  void* v;
+  int sink_held;   // frames in sink slots [0, S)
+  int win_head;    // ring index (0..L-1) of the oldest window frame
+  int win_held;    // frames in the window ring, slots S + (head + i) % L
+  int64_t frames_seen;
+  bool maps_ready;
+  CUtensorMap tm_k, tm_v;
+};
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool desc_ok(const astro_kvcache_desc_t* d) {
+  return d && d->cache_batch >= 1 && d->heads >= 1 && (d->head_dim == 64 || d->head_dim == 128) &&
+         d->tokens_per_frame >= 1 && d->sink_frames >= 0 && d->window_frames >= 1;
+}
+
+// ---- device / driver helpers -------------------------------------------------------------------
+astro_status_t check_arch() {
+  static int ok_device[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ASTRO_ERR_CUDA;
+  if (dev >= 0 && dev < 64 && ok_device[dev]) return ASTRO_OK;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ASTRO_ERR_CUDA;
+  if (major != 10) return ASTRO_ERR_ARCH;
+  if (dev >= 0 && dev < 64) ok_device[dev] = 1;
+  return ASTRO_OK;
+}
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode_fn() {
+  static encode_tiled_fn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<encode_tiled_fn>(p);
+  });
+  return fn;
+}
+
+// bf16 tensor seen as {d, token, head, batch} with byte strides; box = 64 columns x 128 tokens, 128-byte
+// swizzle, zero fill outside the tensor.
+astro_status_t make_tmap(CUtensorMap* out, const void* base, int head_dim, long long n_tok, int heads, int batch,
+                         unsigned long long stride_tok, unsigned long long stride_head,
+                         unsigned long long stride_batch) {
+  encode_tiled_fn fn = get_encode_fn();
+  if (!fn) return ASTRO_ERR_CUDA;
+  cuuint64_t dims[4] = {static_cast<cuuint64_t>(head_dim), static_cast<cuuint64_t>(n_tok),
+                        static_cast<cuuint64_t>(heads), static_cast<cuuint64_t>(batch)};
+  cuuint64_t strides[3] = {stride_tok, stride_head, stride_batch};
+  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(kTile), 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ASTRO_OK : ASTRO_ERR_CUDA;
+}
+
+// Caller tensor [batch, n_tok, H, D].
+astro_status_t make_tmap_user(CUtensorMap* out, const void* base, int head_dim, int n_tok, int heads, int batch) {
+  const unsigned long long row = static_cast<unsigned long long>(head_dim) * 2;
+  return make_tmap(out, base, head_dim, n_tok, heads, batch, row * heads, row, row * heads * n_tok);
+}
+
+astro_status_t ensure_cache_maps(astro_kvcache* c) {
+  if (c->maps_ready) return ASTRO_OK;
+  const auto& d = c->d;
+  const long long tok = static_cast<long long>(d.sink_frames + d.window_frames) * d.tokens_per_frame;
+  const unsigned long long row = static_cast<unsigned long long>(d.head_dim) * 2;
+  astro_status_t s = make_tmap(&c->tm_k, c->k, d.head_dim, tok, d.heads, d.cache_batch, row, row * tok,
+                               row * tok * d.heads);
+  if (s != ASTRO_OK) return s;
+  s = make_tmap(&c->tm_v, c->v, d.head_dim, tok, d.heads, d.cache_batch, row, row * tok, row * tok * d.heads);
+  if (s != ASTRO_OK) return s;
+  c->maps_ready = true;
+  return ASTRO_OK;
+}
+
+// Physical token ranges of the held frames, merged where adjacent, followed by the chunk's keys.
+KeySegs build_segments(const astro_kvcache* c, int n_kc) {
+  KeySegs s;
+  std::memset(&s, 0, sizeof(s));
+  auto push = [&s](long long start, long long count, int from_chunk) {
+    if (count <= 0) return;
+    if (s.n > 0 && !from_chunk && !s.from_chunk[s.n - 1] && s.start[s.n - 1] + s.count[s.n - 1] == start) {
+      s.count[s.n - 1] += static_cast<int>(count);
+      return;
+    }
+    s.start[s.n] = static_cast<int>(start);
+    s.count[s.n] = static_cast<int>(count);
+    s.from_chunk[s.n] = from_chunk;
+    ++s.n;
+  };
+  if (c) {
+    const int T = c->d.tokens_per_frame, S = c->d.sink_frames, L = c->d.window_frames;
+    const int first = c->win_held < L - c->win_head ? c->win_held : L - c->win_head;  // frames before the wrap
+    const int wrapped = c->win_held - first;
+    push(0, static_cast<long long>(c->sink_held) * T, 0);
+    push(static_cast<long long>(S) * T, static_cast<long long>(wrapped) * T, 0);
+    push(static_cast<long long>(S + c->win_head) * T, static_cast<long long>(first) * T, 0);
+  }
+  push(0, n_kc, 1);
+  return s;
+}
+
+template <typename K> astro_status_t set_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess
+             ? ASTRO_OK
+             : ASTRO_ERR_CUDA;
+}
+
+astro_status_t launch_status() { return cudaGetLastError() == cudaSuccess ? ASTRO_OK : ASTRO_ERR_CUDA; }
+
+struct AttnArgs {
+  const astro_kvcache* cache;
+  int batch, heads, head_dim, n_q, n_kc;
+};
+
+astro_status_t check_attn_args(const AttnArgs& a, float scale) {
+  if (a.batch < 1 || a.heads < 1 || a.n_q < 1 || a.n_kc < 0) return ASTRO_ERR_SHAPE;
+  if (a.head_dim != 64 && a.head_dim != 128) return ASTRO_ERR_SHAPE;
+  if (!(scale >= 0.f) || !(scale < 3.0e38f)) return ASTRO_ERR_SHAPE;
+  if (a.batch > 65535 || a.heads > 65535) return ASTRO_ERR_SHAPE;
+  int held = 0;
+  if (a.cache) {
+    const auto& d = a.cache->d;
+    if (d.heads != a.heads || d.head_dim != a.head_dim) return ASTRO_ERR_SHAPE;
+    if (d.cache_batch != a.batch && d.cache_batch != 1) return ASTRO_ERR_SHAPE;
+    held = a.cache->sink_held + a.cache->win_held;
+  }
+  if (held == 0 && a.n_kc == 0) return ASTRO_ERR_SHAPE;  // no key at all: softmax undefined
+  return ASTRO_OK;
+}
+
+template <int D>
+astro_status_t launch_fwd(const AttnArgs& a, const CUtensorMap& tq, const CUtensorMap& tkc, const CUtensorMap& tvc,
+                          const CUtensorMap& tkx, const CUtensorMap& tvx, const KeySegs& segs, float scale, void* o,
+                          float* lse, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    astro_status_t s = set_smem(chunk_attn_fwd_kernel<D>, FwdSmem<D>::kTotal);
+    if (s != ASTRO_OK) return s;
+    attr_set = true;
+  }
+  dim3 grid((a.n_q + kTile - 1) / kTile, a.heads, a.batch);
+  chunk_attn_fwd_kernel<D><<<grid, 128, FwdSmem<D>::kTotal, st>>>(
+      tq, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0,
+      scale * kLog2e, static_cast<__nv_bfloat16*>(o), lse);
+  return launch_status();
+}
+
+template <int D>
+astro_status_t launch_bwd(const AttnArgs& a, const CUtensorMap& tq, const CUtensorMap& tdo, const CUtensorMap& tkc,
+                          const CUtensorMap& tvc, const CUtensorMap& tkx, const CUtensorMap& tvx, const KeySegs& segs,
+                          float scale, const void* o, const float* lse, const void* d_o, float* delta, void* dq,
+                          void* dk, void* dv, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    astro_status_t s = set_smem(chunk_attn_bwd_dq_kernel<D>, BwdSmem<D>::kTotal);
+    if (s != ASTRO_OK) return s;
+    s = set_smem(chunk_attn_bwd_dkv_kernel<D>, BwdSmem<D>::kTotal);
+    if (s != ASTRO_OK) return s;
+    attr_set = true;
+  }
+  const long long rows = static_cast<long long>(a.batch) * a.n_q * a.heads;
+  const unsigned delta_blocks = static_cast<unsigned>((rows * 32 + 255) / 256);
+  bwd_delta_kernel<D><<<delta_blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(o),
+                                                   static_cast<const __nv_bfloat16*>(d_o), delta, a.batch, a.n_q,
+                                                   a.heads);
+  dim3 grid_q((a.n_q + kTile - 1) / kTile, a.heads, a.batch);
+  chunk_attn_bwd_dq_kernel<D><<<grid_q, 128, BwdSmem<D>::kTotal, st>>>(
+      tq, tdo, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads,
+      (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0, scale, lse, delta,
+      static_cast<__nv_bfloat16*>(dq));
+  if (a.n_kc > 0) {
+    dim3 grid_k((a.n_kc + kTile - 1) / kTile, a.heads, a.batch);
+    chunk_attn_bwd_dkv_kernel<D><<<grid_k, 128, BwdSmem<D>::kTotal, st>>>(
+        tq, tdo, tkc, tvc, a.n_q, a.n_kc, a.heads, scale, lse, delta, static_cast<__nv_bfloat16*>(dk),
+        static_cast<__nv_bfloat16*>(dv));
+  }
+  return launch_status();
+}
+
+// Copies frames between a caller tensor and the storage slots listed in `slots` (logical order).
+template <bool ToCache>
+astro_status_t launch_ring_copy(const astro_kvcache* c, void* k_user, void* v_user, const int* slots, int n_frames,
+                                cudaStream_t st) {
+  const auto& d = c->d;
+  const int vpr = d.head_dim * 2 / 16;
+  const long long per_frame = static_cast<long long>(d.tokens_per_frame) * d.heads * vpr;
+  if (per_frame * kMaxFramesPerCopy >= (1ll << 31)) return ASTRO_ERR_SHAPE;
+  for (int f0 = 0; f0 < n_frames; f0 += kMaxFramesPerCopy) {
+    SlotMap map;
+    map.n = n_frames - f0 < kMaxFramesPerCopy ? n_frames - f0 : kMaxFramesPerCopy;
+    for (int j = 0; j < map.n; ++j) map.slot[j] = slots[f0 + j];
+    const long long vec_per_batch = per_frame * map.n;
+    const long long total = vec_per_batch * d.cache_batch;
+    dim3 grid(static_cast<unsigned>((total + 1023) / 1024), 2, 1);
+    ring_copy_kernel<ToCache><<<grid, 256, 0, st>>>(
+        static_cast<uint4*>(k_user), static_cast<uint4*>(v_user), static_cast<uint4*>(c->k),
+        static_cast<uint4*>(c->v), map, d.heads, d.tokens_per_frame, vpr, d.sink_frames + d.window_frames, f0,
+        n_frames, vec_per_batch, total);
+  }
+  return launch_status();
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t astro_kvcache_storage_bytes(const astro_kvcache_desc_t* d) {
+  if (!desc_ok(d)) return 0;
+  return static_cast<size_t>(d->cache_batch) * d->heads * (d->sink_frames + d->window_frames) *
+         d->tokens_per_frame * d->head_dim * 2;
+}
+
+astro_status_t astro_kvcache_create(const astro_kvcache_desc_t* desc, void* k_storage, void* v_storage,
+                                    size_t bytes_each, astro_kvcache_t** out) {
+  if (!desc || !k_storage || !v_storage || !out) return ASTRO_ERR_NULL;
+  if (!desc_ok(desc)) return ASTRO_ERR_SHAPE;
+  if (!aligned16(k_storage) || !aligned16(v_storage)) return ASTRO_ERR_ALIGN;
+  if (bytes_each < astro_kvcache_storage_bytes(desc)) return ASTRO_ERR_CAPACITY;
+  const long long tok = static_cast<long long>(desc->sink_frames + desc->window_frames) * desc->tokens_per_frame;
+  if (tok >= (1ll << 31) - kTile) return ASTRO_ERR_SHAPE;
+  astro_kvcache* c = new (std::nothrow) astro_kvcache();
+  if (!c) return ASTRO_ERR_CUDA;
+  c->d = *desc;
+  c->k = k_storage;
+  c->v = v_storage;
+  c->sink_held = c->win_head = c->win_held = 0;
+  c->frames_seen = 0;
+  c->maps_ready = false;
+  *out = c;
+  return ASTRO_OK;
+}
+
+astro_status_t astro_kvcache_destroy(astro_kvcache_t* cache) {
+  if (!cache) return ASTRO_ERR_NULL;
+  delete cache;
+  return ASTRO_OK;
+}
+
+astro_status_t astro_kvcache_reset(astro_kvcache_t* c) {
+  if (!c) return ASTRO_ERR_NULL;
+  c->sink_held = c->win_head = c->win_held = 0;
+  c->frames_seen = 0;
+  return ASTRO_OK;
+}
+
+astro_status_t astro_kvcache_append(astro_kvcache_t* c, const void* k, const void* v, int n_frames, void* stream) {
+  if (!c || !k || !v) return ASTRO_ERR_NULL;
+  if (n_frames < 0) return ASTRO_ERR_SHAPE;
+  if (!aligned16(k) || !aligned16(v)) return ASTRO_ERR_ALIGN;
+  const int S = c->d.sink_frames, L = c->d.window_frames;
+  const int room = (S - c->sink_held) + (L - c->win_held);
+  if (n_frames > room) return ASTRO_ERR_CAPACITY;
+  if (n_frames == 0) return ASTRO_OK;
+  astro_status_t s = check_arch();
+  if (s != ASTRO_OK) return s;
+  int* slots = new (std::nothrow) int[n_frames];
+  if (!slots) return ASTRO_ERR_CUDA;
+  int sink = c->sink_held, held = c->win_held;
+  for (int j = 0; j < n_frames; ++j) {
+    if (sink < S) slots[j] = sink++;
+    else { slots[j] = S + (c->win_head + held) % L; ++held; }
+  }
+  s = launch_ring_copy<true>(c, const_cast<void*>(k), const_cast<void*>(v), slots, n_frames,
+                             static_cast<cudaStream_t>(stream));
+  delete[] slots;
+  if (s != ASTRO_OK) return s;
+  c->sink_held = sink;
+  c->win_held = held;
+  c->frames_seen += n_frames;
+  return ASTRO_OK;
+}
+
+astro_status_t astro_kvcache_evict(astro_kvcache_t* c, int n_frames, void* /*stream*/) {
+  if (!c) return ASTRO_ERR_NULL;
+  if (n_frames < 0) return ASTRO_ERR_SHAPE;
+  if (n_frames > c->win_held) return ASTRO_ERR_UNDERFLOW;
+  c->win_head = (c->win_head + n_frames) % c->d.window_frames;
+  c->win_held -= n_frames;
+  if (c->win_held == 0) c->win_head = 0;
+  return ASTRO_OK;
+}
+
+astro_status_t astro_kvcache_query(const astro_kvcache_t* c, int* sink_held, int* window_held, int64_t* frames_seen) {
+  if (!c) return ASTRO_ERR_NULL;
+  if (sink_held) *sink_held = c->sink_held;
+  if (window_held) *window_held = c->win_held;
+  if (frames_seen) *frames_seen = c->frames_seen;
+  return ASTRO_OK;
+}
+
+astro_status_t astro_kvcache_export(const astro_kvcache_t* c, void* k_out, void* v_out, void* stream) {
+  if (!c || !k_out || !v_out) return ASTRO_ERR_NULL;
+  if (!aligned16(k_out) || !aligned16(v_out)) return ASTRO_ERR_ALIGN;
+  const int n = c->sink_held + c->win_held;
+  if (n == 0) return ASTRO_OK;
+  astro_status_t s = check_arch();
+  if (s != ASTRO_OK) return s;
+  int* slots = new (std::nothrow) int[n];
+  if (!slots) return ASTRO_ERR_CUDA;
+  for (int j = 0; j < c->sink_held; ++j) slots[j] = j;
+  for (int j = 0; j < c->win_held; ++j)
+    slots[c->sink_held + j] = c->d.sink_frames + (c->win_head + j) % c->d.window_frames;
+  s = launch_ring_copy<false>(c, k_out, v_out, slots, n, static_cast<cudaStream_t>(stream));
+  delete[] slots;
+  return s;
+}
+
+astro_status_t astro_chunk_attn_fwd(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
+                                    const void* v_chunk, int batch, int heads, int head_dim, int n_q, int n_kc,
+                                    float scale, void* o, float* lse, void* stream) {
+  if (!q || !o) return ASTRO_ERR_NULL;
+  if (n_kc > 0 && (!k_chunk || !v_chunk)) return ASTRO_ERR_NULL;
+  const AttnArgs a{cache, batch, heads, head_dim, n_q, n_kc};
+  astro_status_t s = check_attn_args(a, scale);
+  if (s != ASTRO_OK) return s;
+  if (!aligned16(q) || !aligned16(o) || (n_kc > 0 && (!aligned16(k_chunk) || !aligned16(v_chunk))) ||
+      (reinterpret_cast<uintptr_t>(lse) & 3u))
+    return ASTRO_ERR_ALIGN;
+  s = check_arch();
+  if (s != ASTRO_OK) return s;
+  const bool have_ctx = cache && (cache->sink_held + cache->win_held) > 0;
+  CUtensorMap tq, tkc, tvc, tkx, tvx;
+  std::memset(&tkc, 0, sizeof(tkc)); std::memset(&tvc, 0, sizeof(tvc));
+  std::memset(&tkx, 0, sizeof(tkx)); std::memset(&tvx, 0, sizeof(tvx));
+  if ((s = make_tmap_user(&tq, q, head_dim, n_q, heads, batch)) != ASTRO_OK) return s;
+  if (n_kc > 0) {
+    if ((s = make_tmap_user(&tkc, k_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
+    if ((s = make_tmap_user(&tvc, v_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
+  }
+  if (have_ctx) {
+    if ((s = ensure_cache_maps(const_cast<astro_kvcache*>(cache))) != ASTRO_OK) return s;
+    tkx = cache->tm_k;
+    tvx = cache->tm_v;
+  }
+  const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return head_dim == 128 ? launch_fwd<128>(a, tq, tkc, tvc, tkx, tvx, segs, scale, o, lse, st)
+                         : launch_fwd<64>(a, tq, tkc, tvc, tkx, tvx, segs, scale, o, lse, st);
+}
+
+size_t astro_chunk_attn_bwd_workspace_bytes(int batch, int heads, int n_q, int head_dim) {
+  if (batch < 1 || heads < 1 || n_q < 1 || (head_dim != 64 && head_dim != 128)) return 0;
+  const size_t b = static_cast<size_t>(batch) * heads * n_q * sizeof(float);
+  return (b + 255) & ~static_cast<size_t>(255);
+}
+
+astro_status_t astro_chunk_attn_bwd(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
+                                    const void* v_chunk, const void* o, const float* lse, const void* d_o, int batch,
+                                    int heads, int head_dim, int n_q, int n_kc, float scale, void* dq, void* dk_chunk,
+                                    void* dv_chunk, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!q || !o || !lse || !d_o || !dq || !workspace) return ASTRO_ERR_NULL;
+  if (n_kc > 0 && (!k_chunk || !v_chunk || !dk_chunk || !dv_chunk)) return ASTRO_ERR_NULL;
+  const AttnArgs a{cache, batch, heads, head_dim, n_q, n_kc};
+  astro_status_t s = check_attn_args(a, scale);
+  if (s != ASTRO_OK) return s;
+  if (workspace_bytes < astro_chunk_attn_bwd_workspace_bytes(batch, heads, n_q, head_dim)) return ASTRO_ERR_CAPACITY;
+  if (!aligned16(q) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) || !aligned16(workspace) ||
+      (reinterpret_cast<uintptr_t>(lse) & 3u) ||
+      (n_kc > 0 && (!aligned16(k_chunk) || !aligned16(v_chunk) || !aligned16(dk_chunk) || !aligned16(dv_chunk))))
+    return ASTRO_ERR_ALIGN;
+  s = check_arch();
+  if (s != ASTRO_OK) return s;
+  const bool have_ctx = cache && (cache->sink_held + cache->win_held) > 0;
+  CUtensorMap tq, tdo, tkc, tvc, tkx, tvx;
+  std::memset(&tkc, 0, sizeof(tkc)); std::memset(&tvc, 0, sizeof(tvc));
+  std::memset(&tkx, 0, sizeof(tkx)); std::memset(&tvx, 0, sizeof(tvx));
+  if ((s = make_tmap_user(&tq, q, head_dim, n_q, heads, batch)) != ASTRO_OK) return s;
+  if ((s = make_tmap_user(&tdo, d_o, head_dim, n_q, heads, batch)) != ASTRO_OK) return s;
+  if (n_kc > 0) {
+    if ((s = make_tmap_user(&tkc, k_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
+    if ((s = make_tmap_user(&tvc, v_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
+  }
+  if (have_ctx) {
+    if ((s = ensure_cache_maps(const_cast<astro_kvcache*>(cache))) != ASTRO_OK) return s;
+    tkx = cache->tm_k;
+    tvx = cache->tm_v;
+  }
+  const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* delta = static_cast<float*>(workspace);
+  return head_dim == 128 ? launch_bwd<128>(a, tq, tdo, tkc, tvc, tkx, tvx, segs, scale, o, lse, d_o, delta, dq,
+                                           dk_chunk, dv_chunk, st)
+                         : launch_bwd<64>(a, tq, tdo, tkc, tvc, tkx, tvx, segs, scale, o, lse, d_o, delta, dq,
+                                          dk_chunk, dv_chunk, st);
+}
+
+astro_status_t astro_last_device_status(uint32_t* detail) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return ASTRO_ERR_CUDA;
+  uint32_t word = 0;
+  if (cudaMemcpyFromSymbol(&word, g_device_status, sizeof(word)) != cudaSuccess) return ASTRO_ERR_CUDA;
+  if (detail) *detail = word;
+  if (word == 0) return ASTRO_OK;
+  const uint32_t zero = 0;
+  if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)) != cudaSuccess) return ASTRO_ERR_CUDA;
+  return ASTRO_ERR_TIMEOUT;
+}
+
+const char* astro_status_string(astro_status_t s) {
+  switch (s) {
+    case ASTRO_OK: return "ok";
+    case ASTRO_ERR_NULL: return "null pointer";
+    case ASTRO_ERR_SHAPE: return "unsupported or inconsistent shape";
+    case ASTRO_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case ASTRO_ERR_CAPACITY: return "capacity exceeded";
+    case ASTRO_ERR_UNDERFLOW: return "evict exceeds window frames held";
+    case ASTRO_ERR_ARCH: return "device is not compute capability 10.x";
+    case ASTRO_ERR_CUDA: return "CUDA call failed";
+    case ASTRO_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,121 @@
+// Shared pieces of the chunk-attention kernels: the list of key segments a call attends to,
+// the shared-memory tile geometry, and small TMEM/epilogue helpers.
+#pragma once
+#include "sm100_ptx.cuh"
+
+namespace astro {
+
+constexpr int kTile = 128;  // query rows per CTA tile and keys per key tile
+
+// The keys of one call: up to two contiguous token ranges of the cache storage (the ring can be
+// split by its wrap-around or by a hole left by evict) and the chunk's own keys.
+struct KeySegs {
+  int n;
+  int start[3];     // first token (row of the source tensor)
+  int count[3];     // tokens in the segment (> 0)
+  int from_chunk[3];  // 1: rows of K_chunk/V_chunk, 0: rows of the cache storage
+};
+
+__host__ __device__ inline int seg_tiles(const KeySegs& s) {
+  int t = 0;
+  for (int i = 0; i < s.n; ++i) t += (s.count[i] + kTile - 1) / kTile;
+  return t;
+}
+
+// Walks key tiles segment by segment.
+struct KeyTileIter {
+  int seg, off;
+  __device__ KeyTileIter() : seg(0), off(0) {}
+  __device__ bool done(const KeySegs& s) const { return seg >= s.n; }
+  __device__ int row0(const KeySegs& s) const { return s.start[seg] + off; }
+  __device__ int valid(const KeySegs& s) const { return min(kTile, s.count[seg] - off); }
+  __device__ int from_chunk(const KeySegs& s) const { return s.from_chunk[seg]; }
+  __device__ void next(const KeySegs& s) {
+    off += kTile;
+    if (off >= s.count[seg]) { ++seg; off = 0; }
+  }
+};
+
+// A [128 x D] bf16 tile sits in shared memory as D/64 blocks of [128 rows x 128 bytes], 128-byte
+// swizzled by TMA; block h holds columns 64h..64h+63.
+template <int D> struct TileGeom {
+  static constexpr int kBlocks = D / 64;
+  static constexpr int kBlockBytes = kTile * 128;
+  static constexpr int kBytes = kBlocks * kBlockBytes;
+};
+
+template <int D>
+__device__ __forceinline__ void tma_load_tile(uint8_t* smem_tile, const CUtensorMap* tm, uint64_t* bar, int row0,
+                                              int h, int b) {
+#pragma unroll
+  for (int blk = 0; blk < TileGeom<D>::kBlocks; ++blk)
+    tma_load_4d(smem_tile + blk * TileGeom<D>::kBlockBytes, tm, bar, blk * 64, row0, h, b);
+}
+
+// acc[128 x 128] = A[128 x D] * B[128 x D]^T, both tiles K-major (contraction over D).
+template <int D>
+__device__ __forceinline__ void mma_abT(uint32_t d_tmem, uint32_t a_smem, uint32_t b_smem) {
+  constexpr uint32_t idesc = make_idesc_bf16(kTile, kTile, false, false);
+#pragma unroll
+  for (int k = 0; k < D / 16; ++k) {
+    const uint32_t off = (k >> 2) * TileGeom<D>::kBlockBytes + (k & 3) * 32;
+    mma_ss(d_tmem, desc_kmajor(a_smem + off), desc_kmajor(b_smem + off), idesc, k > 0);
+  }
+}
+
+// acc[128 x D] (+)= A_tmem[128 x 128 bf16] * B[128 x D] with the contraction over B's rows (MN-major B).
+template <int D>
+__device__ __forceinline__ void mma_pb(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_smem, bool accumulate) {
+  constexpr uint32_t idesc = make_idesc_bf16(kTile, D, false, true);
+#pragma unroll
+  for (int k = 0; k < kTile / 16; ++k)
+    mma_ts(d_tmem, a_tmem + k * 8, desc_mnmajor(b_smem + k * 2048, TileGeom<D>::kBlockBytes), idesc,
+           (accumulate || k > 0) ? 1u : 0u);
+}
+
+// Zero rows [first_row, 128) of a tile in shared memory (every block), then publish to the async proxy.
+// Row r of a block occupies bytes [128 r, 128 r + 128) whatever the swizzle.  Called by 128 threads.
+template <int D>
+__device__ __forceinline__ void zero_tile_rows_from(uint8_t* smem_tile, int first_row, int tid) {
+  if (tid >= first_row) {
+#pragma unroll
+    for (int blk = 0; blk < TileGeom<D>::kBlocks; ++blk) {
+      uint4* p = reinterpret_cast<uint4*>(smem_tile + blk * TileGeom<D>::kBlockBytes + tid * 128);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) p[i] = make_uint4(0, 0, 0, 0);
+    }
+  }
+  fence_proxy_async_smem();
+}
+
+// Write one row of D fp32 accumulators (TMEM columns [col0, col0+D) of this thread's lane), times
+// `mult`, as bf16 to `dst` (global, 16-byte aligned) when `store` is set.  Warp-collective.
+template <int D>
+__device__ __forceinline__ void store_row_from_tmem(uint32_t taddr_lane_col0, float mult, __nv_bfloat16* dst,
+                                                    bool store) {
+#pragma unroll
+  for (int j = 0; j < D / 32; ++j) {
+    uint32_t r[32];
+    tmem_ld32(taddr_lane_col0 + j * 32, r);
+    tmem_wait_ld();
+    if (store) {
+      uint4* out = reinterpret_cast<uint4*>(dst + j * 32);
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        uint4 w;
+        w.x = pack_bf16(__uint_as_float(r[8 * v + 0]) * mult, __uint_as_float(r[8 * v + 1]) * mult);
+        w.y = pack_bf16(__uint_as_float(r[8 * v + 2]) * mult, __uint_as_float(r[8 * v + 3]) * mult);
+        w.z = pack_bf16(__uint_as_float(r[8 * v + 4]) * mult, __uint_as_float(r[8 * v + 5]) * mult);
+        w.w = pack_bf16(__uint_as_float(r[8 * v + 6]) * mult, __uint_as_float(r[8 * v + 7]) * mult);
+        out[v] = w;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ uint8_t* align_1024(uint8_t* p) {
+  const uint32_t a = smem_u32(p);
+  return p + ((1024u - (a & 1023u)) & 1023u);
+}
+
+}  // namespace astro
