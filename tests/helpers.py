@@ -24,10 +24,10 @@ def rel_l2(got, ref):
 O_MAX_ABS, O_MEAN_ABS, LSE_ABS, GRAD_REL_L2 = 1e-2, 1e-3, 1e-3, 1e-2
 
 
-def check_fwd(o, lse, o_ref, lse_ref, tag=""):
+def check_fwd(o, lse, o_ref, lse_ref, tag="", o_max_abs=O_MAX_ABS, o_mean_abs=O_MEAN_ABS):
     d = np.abs(f64(o) - o_ref)
-    assert d.max() <= O_MAX_ABS, "%s O max-abs %.3e" % (tag, d.max())
-    assert d.mean() <= O_MEAN_ABS, "%s O mean-abs %.3e" % (tag, d.mean())
+    assert d.max() <= o_max_abs, "%s O max-abs %.3e" % (tag, d.max())
+    assert d.mean() <= o_mean_abs, "%s O mean-abs %.3e" % (tag, d.mean())
     dl = np.abs(f64(lse) - lse_ref)
     assert dl.max() <= LSE_ABS, "%s LSE abs %.3e" % (tag, dl.max())
 
@@ -36,5 +36,8 @@ def check_grads(got, ref, tag=""):
     for g, r, name in zip(got, ref, ("dQ", "dK", "dV")):
         if g is None:
             continue
-        e = rel_l2(f64(g), r)
-        assert e <= GRAD_REL_L2, "%s %s rel-L2 %.3e" % (tag, name, e)
+        # relative L2 with an absolute floor of 1e-6 per element, for gradients that are exactly zero
+        # mathematically (a single key: softmax is constant, dQ = dK = 0) where fp32 rounding noise remains
+        err = float(np.linalg.norm(f64(g) - r))
+        bound = GRAD_REL_L2 * float(np.linalg.norm(r)) + 1e-6 * np.sqrt(r.size)
+        assert err <= bound, "%s %s rel-L2 %.3e (err %.3e, bound %.3e)" % (tag, name, rel_l2(f64(g), r), err, bound)

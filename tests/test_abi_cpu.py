@@ -1,0 +1,115 @@
+"""CPU-side checks of the C ABI: the library builds, loads and exports what include/astro.h declares,
+and host-only argument validation and ring metadata behave as documented (no kernel is launched)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2603_17051_b200 import binding as A
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "astro.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(astro_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    L = A.lib()
+    names = declared_functions()
+    assert len(names) >= 13
+    for n in names:
+        assert hasattr(L, n), n
+    assert sorted(A.EXPORTED) == [n for n in names if n in A.EXPORTED]
+    assert set(names) == set(A.EXPORTED)
+
+
+def test_status_strings():
+    seen = set()
+    for code in range(9):
+        s = A.status_string(code)
+        assert s and s != "unknown status"
+        seen.add(s)
+    assert len(seen) == 9
+    assert A.status_string(99) == "unknown status"
+
+
+def test_storage_and_workspace_bytes():
+    assert A.astro_kvcache_storage_bytes(1, 12, 128, 1560, 3, 18) == 12 * 21 * 1560 * 128 * 2
+    assert A.astro_kvcache_storage_bytes(4, 12, 128, 1560, 3, 12) == 4 * 12 * 15 * 1560 * 128 * 2
+    assert A.astro_kvcache_storage_bytes(1, 12, 96, 1560, 3, 18) == 0      # head_dim must be 64 or 128
+    assert A.astro_kvcache_storage_bytes(1, 12, 128, 1560, 3, 0) == 0       # window needs a slot
+    assert A.astro_chunk_attn_bwd_workspace_bytes(2, 12, 4680, 128) == 2 * 12 * 4680 * 4 + (-(2 * 12 * 4680 * 4)) % 256
+    assert A.astro_chunk_attn_bwd_workspace_bytes(2, 12, 4680, 100) == 0
+
+
+def _raw_create(desc, k=0x10000, v=0x20000, nbytes=1 << 40):
+    out = C.c_void_p()
+    st = A.lib().astro_kvcache_create(C.byref(desc) if desc is not None else None, C.c_void_p(k), C.c_void_p(v),
+                                      nbytes, C.byref(out))
+    return st, out
+
+
+def test_create_validation_and_ring_metadata_without_a_device():
+    L = A.lib()
+    d = A.KVCacheDesc(1, 2, 64, 16, 1, 4)
+    assert _raw_create(None)[0] == 1
+    assert _raw_create(d, k=0)[0] == 1
+    assert _raw_create(A.KVCacheDesc(1, 2, 80, 16, 1, 4))[0] == 2
+    assert _raw_create(d, k=0x10008)[0] == 3
+    assert _raw_create(d, nbytes=100)[0] == 4
+    st, h = _raw_create(d)
+    assert st == 0
+    a, b, c = C.c_int(-1), C.c_int(-1), C.c_int64(-1)
+    assert L.astro_kvcache_query(h, C.byref(a), C.byref(b), C.byref(c)) == 0
+    assert (a.value, b.value, c.value) == (0, 0, 0)
+    # evict on an empty window underflows; negative counts are shape errors; zero is fine
+    assert L.astro_kvcache_evict(h, 1, None) == 5
+    assert L.astro_kvcache_evict(h, -1, None) == 2
+    assert L.astro_kvcache_evict(h, 0, None) == 0
+    # capacity is checked before anything touches the device: S+L = 5 frames
+    assert L.astro_kvcache_append(h, C.c_void_p(0x30000), C.c_void_p(0x40000), 6, None) == 4
+    assert L.astro_kvcache_append(h, None, C.c_void_p(0x40000), 1, None) == 1
+    assert L.astro_kvcache_append(h, C.c_void_p(0x30004), C.c_void_p(0x40000), 1, None) == 3
+    assert L.astro_kvcache_append(h, C.c_void_p(0x30000), C.c_void_p(0x40000), 0, None) == 0
+    assert L.astro_kvcache_reset(h) == 0
+    assert L.astro_kvcache_destroy(h) == 0
+    assert L.astro_kvcache_destroy(None) == 1
+
+
+def test_attention_argument_validation_happens_before_any_launch():
+    L = A.lib()
+    p = C.c_void_p(0x10000)
+    lse = C.c_void_p(0x50000)
+    # no key at all
+    assert L.astro_chunk_attn_fwd(None, p, None, None, 1, 2, 64, 48, 0, 0.125, p, lse, None) == 2
+    # unsupported head_dim, negative scale, null q
+    assert L.astro_chunk_attn_fwd(None, p, p, p, 1, 2, 96, 48, 48, 0.125, p, lse, None) == 2
+    assert L.astro_chunk_attn_fwd(None, p, p, p, 1, 2, 64, 48, 48, -1.0, p, lse, None) == 2
+    assert L.astro_chunk_attn_fwd(None, None, p, p, 1, 2, 64, 48, 48, 0.125, p, lse, None) == 1
+    assert L.astro_chunk_attn_fwd(None, C.c_void_p(0x10002), p, p, 1, 2, 64, 48, 48, 0.125, p, lse, None) == 3
+    # cache with other head count / batch
+    st, h = _raw_create(A.KVCacheDesc(2, 2, 64, 16, 0, 4))
+    assert st == 0
+    assert L.astro_chunk_attn_fwd(h, p, p, p, 3, 2, 64, 48, 48, 0.125, p, lse, None) == 2
+    assert L.astro_chunk_attn_fwd(h, p, p, p, 2, 4, 64, 48, 48, 0.125, p, lse, None) == 2
+    # backward: workspace too small, null dO
+    assert L.astro_chunk_attn_bwd(None, p, p, p, p, lse, p, 1, 2, 64, 48, 48, 0.125, p, p, p, p, 16, None) == 4
+    assert L.astro_chunk_attn_bwd(None, p, p, p, p, lse, None, 1, 2, 64, 48, 48, 0.125, p, p, p, p, 4096, None) == 1
+    L.astro_kvcache_destroy(h)
+
+
+def test_product_never_reaches_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2603_17051_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert not re.search(r"^\s*(from|import)\s+oracle|#include.*oracle|oracle[./]", text, flags=re.M), f
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith(".py"):
+            text = open(os.path.join(ROOT, "oracle", f)).read()
+            assert "paper_2603_17051_b200" not in text and "ctypes" not in text, f

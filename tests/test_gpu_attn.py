@@ -1,0 +1,237 @@
+"""GPU parity of chunk attention forward and backward against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from helpers import check_fwd, check_grads, dev_bf16, f64, host_bits, rel_l2
+from oracle import rolling_attn as orc
+from paper_2603_17051_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _ctx(model):
+    mk, mv = model.export()
+    if mk is None:
+        return None, None
+    return orc.bf16_bits_to_f64(mk), orc.bf16_bits_to_f64(mv)
+
+
+def _fill(A, Bc, H, D, T, S, L, held, seed, churn=0):
+    """Cache + model holding `held` frames; `churn` extra evict/append rounds move the ring head."""
+    cache = A.astro_kvcache_create(Bc, H, D, T, S, L)
+    model = orc.RollingKVCache(S, L)
+    if held:
+        kb = synth.normal_bf16(seed, (Bc, held * T, H, D)); vb = synth.normal_bf16(seed + 1, (Bc, held * T, H, D))
+        A.astro_kvcache_append(cache, dev_bf16(kb), dev_bf16(vb), held); model.append(kb, vb, T)
+    for r in range(churn):
+        n = min(2, len(model.win_k))
+        if n == 0:
+            break
+        A.astro_kvcache_evict(cache, n); model.evict(n)
+        kb = synth.normal_bf16(seed + 10 + 2 * r, (Bc, n * T, H, D)); vb = synth.normal_bf16(seed + 11 + 2 * r, (Bc, n * T, H, D))
+        A.astro_kvcache_append(cache, dev_bf16(kb), dev_bf16(vb), n); model.append(kb, vb, T)
+    return cache, model
+
+
+def _run_case(A, B, Bc, H, D, T, S, L, held, n_q, n_kc, seed, churn=0, evict_hole=0, scale=None, bwd=True,
+              o_max_abs=1e-2, o_mean_abs=1e-3):
+    scale = 1.0 / np.sqrt(D) if scale is None else scale
+    cache, model = _fill(A, Bc, H, D, T, S, L, held, seed, churn)
+    if evict_hole:
+        A.astro_kvcache_evict(cache, evict_hole); model.evict(evict_hole)
+    bits = [synth.normal_bf16(seed + 100 + i, shp) for i, shp in
+            enumerate(((B, n_q, H, D), (B, n_kc, H, D), (B, n_kc, H, D), (B, n_q, H, D)))]
+    q, kc, vc, do = (dev_bf16(x) for x in bits)
+    qf, kf, vf, dof = (orc.bf16_bits_to_f64(x) for x in bits)
+    if n_kc == 0:
+        kc = vc = None
+    kx, vx = _ctx(model)
+    o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, scale)
+    A.astro_last_device_status()
+    o_ref, lse_ref = orc.chunk_attn_fwd(qf, kx, vx, kf, vf, scale)
+    check_fwd(o, lse, o_ref, lse_ref, o_max_abs=o_max_abs, o_mean_abs=o_mean_abs)
+    if bwd:
+        g = A.astro_chunk_attn_bwd(cache, q, kc, vc, o, lse, do, scale)
+        A.astro_last_device_status()
+        g_ref = orc.chunk_attn_bwd(qf, kx, vx, kf, vf, dof, scale)
+        check_grads(g, g_ref)
+    return cache, model
+
+
+def test_tiny_config_streamed_four_chunks():
+    """The tiny workload end to end: 4 chunks with evict/append, forward and backward each chunk, exhaustive."""
+    from paper_2603_17051_b200 import binding as A
+    w = synth.TINY
+    cache = A.astro_kvcache_create(w.cache_batch, w.heads, w.head_dim, w.tokens_per_frame, w.sink_frames, w.window_frames)
+    model = orc.RollingKVCache(w.sink_frames, w.window_frames)
+    M = w.chunk_tokens
+    for n in range(4):
+        over = model.held() - (w.sink_frames + w.window_frames - w.chunk_frames)
+        if over > 0:
+            A.astro_kvcache_evict(cache, over); model.evict(over)
+        bits = [synth.normal_bf16(synth.tensor_seed(1, 10 * n + i), (w.batch, M, w.heads, w.head_dim)) for i in range(4)]
+        q, kc, vc, do = (dev_bf16(x) for x in bits)
+        qf, kf, vf, dof = (orc.bf16_bits_to_f64(x) for x in bits)
+        kx, vx = _ctx(model)
+        o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, w.scale)
+        g = A.astro_chunk_attn_bwd(cache, q, kc, vc, o, lse, do, w.scale)
+        A.astro_last_device_status()
+        check_fwd(o, lse, *orc.chunk_attn_fwd(qf, kx, vx, kf, vf, w.scale), tag="chunk %d" % n)
+        check_grads(g, orc.chunk_attn_bwd(qf, kx, vx, kf, vf, dof, w.scale), tag="chunk %d" % n)
+        A.astro_kvcache_append(cache, kc, vc, w.chunk_frames); model.append(bits[1], bits[2], w.tokens_per_frame)
+        ke, ve = A.astro_kvcache_export(cache)
+        mk, mv = model.export()
+        assert np.array_equal(host_bits(ke), mk) and np.array_equal(host_bits(ve), mv)
+
+
+@pytest.mark.parametrize("case", [
+    # several tiles with ragged tails everywhere, per-sample caches, wrapped ring
+    dict(B=2, Bc=2, H=3, D=128, T=100, S=1, L=5, held=6, n_q=300, n_kc=300, seed=100, churn=2),
+    # shared frozen prefix (B_c = 1) broadcast over a group of 3
+    dict(B=3, Bc=1, H=2, D=128, T=50, S=2, L=6, held=8, n_q=333, n_kc=77, seed=200, churn=3),
+    # head_dim 64, a hole left by evict without re-append
+    dict(B=1, Bc=1, H=2, D=64, T=33, S=1, L=7, held=8, n_q=130, n_kc=99, seed=300, churn=2, evict_hole=3),
+    # no cached context at all; n_q != n_kc
+    dict(B=2, Bc=2, H=2, D=128, T=16, S=0, L=2, held=0, n_q=200, n_kc=129, seed=400),
+    # context only, no chunk keys
+    dict(B=1, Bc=1, H=2, D=64, T=40, S=0, L=5, held=5, n_q=64, n_kc=0, seed=500),
+    # one query, one key
+    dict(B=1, Bc=1, H=1, D=64, T=1, S=0, L=1, held=0, n_q=1, n_kc=1, seed=600),
+    # sink only partly filled
+    dict(B=1, Bc=1, H=1, D=128, T=10, S=4, L=3, held=2, n_q=17, n_kc=5, seed=700),
+    # exact multiples of the tile
+    dict(B=1, Bc=1, H=2, D=128, T=128, S=1, L=3, held=4, n_q=256, n_kc=256, seed=800, churn=1),
+    # a scale other than 1/sqrt(D): near one-hot softmax, the running max moves.  O is then about one V row
+    # (|v| up to ~4.5), so the bf16 rounding of P (2^-9 relative) and of O (half an ulp, 2^-9 |o|) bound the
+    # error by 2^-8 max|v| = 1.8e-2 rather than by the 1e-2 of the 1/sqrt(D) workloads; the mean error of
+    # rounding a unit-magnitude output to bf16 alone is about a quarter ulp, 2^-9.5 E|o| = 1.1e-3, so 2.5e-3.
+    dict(B=1, Bc=1, H=2, D=128, T=64, S=0, L=6, held=6, n_q=200, n_kc=100, seed=900, scale=0.7, o_max_abs=1.8e-2,
+         o_mean_abs=2.5e-3),
+])
+def test_parity_cases(case):
+    from paper_2603_17051_b200 import binding as A
+    _run_case(A, **case)
+
+
+def test_single_key_and_identical_keys_closed_forms_on_gpu():
+    import torch
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, n_q = 1, 2, 64, 70
+    q = dev_bf16(synth.normal_bf16(1, (B, n_q, H, D)))
+    v1 = dev_bf16(synth.normal_bf16(2, (B, 1, H, D))); k1 = dev_bf16(synth.normal_bf16(3, (B, 1, H, D)))
+    o, lse = A.astro_chunk_attn_fwd(None, q, k1, v1, 0.125)
+    assert torch.equal(o, v1.expand(B, n_q, H, D))                      # one key: O is its V, exactly
+    kk = k1.expand(B, 37, H, D).contiguous()
+    vv = dev_bf16(synth.normal_bf16(4, (B, 37, H, D)))
+    o, lse2 = A.astro_chunk_attn_fwd(None, q, kk, vv, 0.125)
+    assert (o.float() - vv.float().mean(1, keepdim=True)).abs().max() < 1e-2
+    assert (lse2 - (lse + float(np.log(37)))).abs().max() < 1e-3
+
+
+def test_shared_prefix_equals_replicated_caches():
+    import torch
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, T, S, L, held = 3, 2, 128, 30, 1, 4, 5
+    c1 = A.astro_kvcache_create(1, H, D, T, S, L); cB = A.astro_kvcache_create(B, H, D, T, S, L)
+    k = dev_bf16(synth.normal_bf16(11, (1, held * T, H, D))); v = dev_bf16(synth.normal_bf16(12, (1, held * T, H, D)))
+    A.astro_kvcache_append(c1, k, v, held)
+    A.astro_kvcache_append(cB, k.expand(B, -1, -1, -1).contiguous(), v.expand(B, -1, -1, -1).contiguous(), held)
+    q, kc, vc, do = (dev_bf16(synth.normal_bf16(13 + i, (B, 90, H, D))) for i in range(4))
+    o1, l1 = A.astro_chunk_attn_fwd(c1, q, kc, vc, 0.1)
+    oB, lB = A.astro_chunk_attn_fwd(cB, q, kc, vc, 0.1)
+    assert torch.equal(o1, oB) and torch.equal(l1, lB)
+    g1 = A.astro_chunk_attn_bwd(c1, q, kc, vc, o1, l1, do, 0.1)
+    gB = A.astro_chunk_attn_bwd(cB, q, kc, vc, oB, lB, do, 0.1)
+    for a, b in zip(g1, gB):
+        assert torch.equal(a, b)
+
+
+def test_stale_nan_in_evicted_slots_does_not_leak():
+    """Tile rows past a segment's end may hold anything (here NaN): results must not change."""
+    import torch
+    from paper_2603_17051_b200 import binding as A
+    H, D, T, S, L = 2, 128, 50, 0, 4
+    cache = A.astro_kvcache_create(1, H, D, T, S, L)
+    cache.k_storage.view(torch.int16).fill_(0x7FC0 - 0x10000 if False else 0x7FC0)
+    cache.v_storage.view(torch.int16).fill_(0x7FC0)
+    model = orc.RollingKVCache(S, L)
+    kb = synth.normal_bf16(21, (1, 3 * T, H, D)); vb = synth.normal_bf16(22, (1, 3 * T, H, D))
+    A.astro_kvcache_append(cache, dev_bf16(kb), dev_bf16(vb), 3); model.append(kb, vb, T)
+    bits = [synth.normal_bf16(23 + i, (1, 60, H, D)) for i in range(4)]
+    q, kc, vc, do = (dev_bf16(x) for x in bits)
+    qf, kf, vf, dof = (orc.bf16_bits_to_f64(x) for x in bits)
+    o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, 0.09)
+    g = A.astro_chunk_attn_bwd(cache, q, kc, vc, o, lse, do, 0.09)
+    kx, vx = _ctx(model)
+    check_fwd(o, lse, *orc.chunk_attn_fwd(qf, kx, vx, kf, vf, 0.09))
+    check_grads(g, orc.chunk_attn_bwd(qf, kx, vx, kf, vf, dof, 0.09))
+
+
+def test_canary_padding_around_outputs_is_untouched():
+    import torch
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, n_q, n_kc = 1, 2, 128, 150, 140
+    pad = 4096
+    def padded(shape, dtype):
+        n = int(np.prod(shape))
+        buf = torch.full((n + 2 * pad,), 7, dtype=dtype, device="cuda")
+        return buf, buf[pad:pad + n].view(shape)
+    q, kc, vc, do = (dev_bf16(synth.normal_bf16(31 + i, (B, n, H, D))) for i, n in enumerate((n_q, n_kc, n_kc, n_q)))
+    ob, o = padded((B, n_q, H, D), torch.bfloat16); lb, lse = padded((B, H, n_q), torch.float32)
+    A.astro_chunk_attn_fwd(None, q, kc, vc, 0.1, o=o, lse=lse)
+    dqb, dq = padded((B, n_q, H, D), torch.bfloat16); dkb, dk = padded((B, n_kc, H, D), torch.bfloat16)
+    dvb, dv = padded((B, n_kc, H, D), torch.bfloat16)
+    A.astro_chunk_attn_bwd(None, q, kc, vc, o, lse, do, 0.1, dq=dq, dk_chunk=dk, dv_chunk=dv)
+    A.astro_last_device_status()
+    for buf in (ob, lb, dqb, dkb, dvb):
+        assert (buf[:pad] == 7).all() and (buf[-pad:] == 7).all()
+
+
+def _sample_rows(n_q, n_rand, rng):
+    tail = np.arange((n_q // 128) * 128, n_q)                       # every row of the ragged last tile
+    rows = np.unique(np.concatenate([rng.choice(n_q, n_rand, replace=False), tail, [0, 127, 128]]))
+    return rows
+
+
+def test_layer_shape_forward_sampled_rows():
+    """Full-size single-layer forward (12 heads, D=128, 4680 queries x 32760 keys) in the launch
+    configuration the benchmark times; the oracle computes sampled query rows one by one."""
+    from paper_2603_17051_b200 import binding as A
+    w = synth.LAYER_FWD
+    cache, model = _fill(A, w.cache_batch, w.heads, w.head_dim, w.tokens_per_frame, w.sink_frames,
+                         w.window_frames, w.held_frames, synth.tensor_seed(2, 0), churn=2)
+    bits = [synth.normal_bf16(synth.tensor_seed(2, 50 + i), (w.batch, w.chunk_tokens, w.heads, w.head_dim)) for i in range(3)]
+    q, kc, vc = (dev_bf16(x) for x in bits)
+    o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, w.scale)
+    A.astro_last_device_status()
+    rows = _sample_rows(w.chunk_tokens, 64, np.random.default_rng(2))
+    kx, vx = _ctx(model)
+    qf, kf, vf = (orc.bf16_bits_to_f64(x) for x in bits)
+    o_ref, lse_ref = orc.chunk_attn_fwd(qf[:, rows], kx, vx, kf, vf, w.scale)
+    check_fwd(o[:, rows], lse[:, :, rows], o_ref, lse_ref)
+
+
+def test_rl_update_shape_backward_sampled():
+    """Full-size clip-window update (batch 2, 28080 detached keys + 4680 trainable): dQ on sampled rows
+    (rows are independent), dK/dV in full for two (sample, head) pairs."""
+    from paper_2603_17051_b200 import binding as A
+    w = synth.RL_UPDATE
+    cache, model = _fill(A, w.cache_batch, w.heads, w.head_dim, w.tokens_per_frame, w.sink_frames,
+                         w.window_frames, w.held_frames, synth.tensor_seed(4, 0), churn=1)
+    bits = [synth.normal_bf16(synth.tensor_seed(4, 50 + i), (w.batch, w.chunk_tokens, w.heads, w.head_dim)) for i in range(4)]
+    q, kc, vc, do = (dev_bf16(x) for x in bits)
+    o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, w.scale)
+    dq, dk, dv = A.astro_chunk_attn_bwd(cache, q, kc, vc, o, lse, do, w.scale)
+    A.astro_last_device_status()
+    mk, mv = model.export()
+    rows = _sample_rows(w.chunk_tokens, 48, np.random.default_rng(4))
+    for (b, h) in ((0, 3), (1, 11)):
+        sl = lambda x: orc.bf16_bits_to_f64(x[b:b + 1, :, h:h + 1, :])
+        qf, kf, vf, dof, kx, vx = sl(bits[0]), sl(bits[1]), sl(bits[2]), sl(bits[3]), sl(mk), sl(mv)
+        o_ref, lse_ref = orc.chunk_attn_fwd(qf, kx, vx, kf, vf, w.scale)
+        check_fwd(o[b:b + 1, :, h:h + 1], lse[b:b + 1, h:h + 1], o_ref, lse_ref, tag="b%d h%d" % (b, h))
+        dq_ref, dk_ref, dv_ref = orc.chunk_attn_bwd(qf, kx, vx, kf, vf, dof, w.scale)
+        check_grads((dq[b:b + 1, :, h:h + 1], dk[b:b + 1, :, h:h + 1], dv[b:b + 1, :, h:h + 1]),
+                    (dq_ref, dk_ref, dv_ref), tag="b%d h%d" % (b, h))
+        e = rel_l2(f64(dq[b:b + 1, rows, h:h + 1]), dq_ref[:, rows])
+        assert e <= 1e-2, "sampled dQ rows rel-L2 %.3e" % e
