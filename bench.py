@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of rolling-KV chunk attention on the single-layer 1.3B-class shape.
+
+One step = one pass of the whole hot path on one batch of synthetic input:
+evict 3 frames, forward (O, LSE) of a 3-frame chunk (4680 queries) against 18 held
+frames + the chunk (32760 keys), backward (delta, dQ, dK/dV of the chunk), append the
+chunk's K/V.  12 heads, head_dim 128, 1560 tokens per latent frame, bf16, scale 1/sqrt(D).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  With N > 1 (under torchrun) every rank runs an independent
+replica of the step on its own GPU (the path has no exchange step); the time is the
+maximum over ranks and the value the sum of the work.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2603_17051_b200 import synth
+
+METRIC = "chunk_attn_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+W = synth.LAYER_FWD
+WORKLOAD = ("layer_fwd shape + backward: B=1 H=12 D=128 T=1560, chunk 3 frames (4680 q), 18 held frames + chunk = "
+            "32760 keys, S=3 sink + 18 window slots; step = evict 3, fwd, bwd (delta+dQ+dK/dV), append 3")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16_burst": float(p["bf16_tflops"]), "bf16_sustained": float(p["bf16_tflops_sustained"]),
+                "hbm": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm": 6650.0, "source": "fallback"}
+
+
+def rank_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Largest value any rank holds (the job is as slow as its slowest rank)."""
+    if world == 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate(flops_per_rank_step: float, ms_per_step_max: float, world: int) -> float:
+    """Whole-job TFLOP/s of `world` independent replicas whose slowest one takes ms_per_step_max."""
+    return world * flops_per_rank_step / (ms_per_step_max * 1e-3) / 1e12
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.gpu_id = gpu_id
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        mhz, mx, reasons = [], None, set()
+        for ts, line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6 or not (t0 <= ts <= t1 + 0.05):
+                continue
+            try:
+                mhz.append(float(parts[0])); mx = float(parts[1])
+            except ValueError:
+                continue
+            for name, val in zip(self.NAMES, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not mhz:  # region shorter than the sampling period: take whatever was seen
+            for ts, line in self.lines:
+                parts = [p.strip() for p in line.split(",")]
+                try:
+                    mhz.append(float(parts[0])); mx = float(parts[1])
+                except (ValueError, IndexError):
+                    pass
+        return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(mhz)}
+
+
+# ----------------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample_inputs(n_rows: int):
+    """One head of the workload, `n_rows` query rows: bf16-rounded N(0,1) widened to fp64."""
+    from oracle import rolling_attn as orc
+    D = W.head_dim
+    mk = lambda i, n: orc.bf16_bits_to_f64(synth.normal_bf16(synth.tensor_seed(2, 900 + i), (1, n, 1, D)))
+    return (mk(0, n_rows), mk(1, W.ctx_tokens), mk(2, W.ctx_tokens), mk(3, W.chunk_tokens), mk(4, W.chunk_tokens),
+            mk(5, n_rows))
+
+
+def oracle_step(inp):
+    from oracle import rolling_attn as orc
+    q, kx, vx, kc, vc, do = inp
+    o, lse = orc.chunk_attn_fwd(q, kx, vx, kc, vc, W.scale)
+    orc.bwd_delta(o, do)
+    return orc.chunk_attn_bwd(q, kx, vx, kc, vc, do, W.scale)
+
+
+def sample_flops(n_rows: int) -> float:
+    D, nk, nkc = W.head_dim, W.total_keys, W.chunk_tokens
+    return n_rows * D * (4.0 * nk + 6.0 * nk + 4.0 * nkc)
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return int(max(n)) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(n_rows: int, reps: int):
+    inp = oracle_sample_inputs(n_rows)
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle_step(inp)
+    dt = (time.perf_counter() - t0) / reps
+    return sample_flops(n_rows) / dt / 1e12, dt
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, timed on the host cores, on a bounded sample of the same workload."""
+    rank, _, world = rank_env()
+    if rank != 0:
+        return 0
+    n_rows = 256
+    sample = "1 of 12 heads x %d of 4680 query rows against all 32760 keys, fwd+bwd, fp64 numpy" % n_rows
+    inp = oracle_sample_inputs(n_rows)
+    for _ in range(args.warmup):
+        oracle_step(inp)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(inp)
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    val = sample_flops(n_rows) / dt / 1e12
+    cores = blas_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "note": "each step is the bounded sample below, not the whole workload"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import torch
+    from paper_2603_17051_b200 import binding as A
+
+    rank, local_rank, world = rank_env()
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank if world > 1 else 0)
+    torch.cuda.set_device(dev)
+    peaks = measured_peaks()
+    B, H, D, T, M = W.batch, W.heads, W.head_dim, W.tokens_per_frame, W.chunk_tokens
+    c = W.chunk_frames
+
+    def host_normal(i, shape):
+        bits = synth.normal_bf16(synth.tensor_seed(2, 100 * rank + i), shape)
+        return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+
+    # inputs: resident copies for the device-timed arm, pinned host copies for the end-to-end arm
+    h_q, h_kc, h_vc, h_do = (host_normal(i, (B, M, H, D)).pin_memory() for i in range(4))
+    q, kc, vc, do = (t.to(dev) for t in (h_q, h_kc, h_vc, h_do))
+    cache = A.astro_kvcache_create(W.cache_batch, H, D, T, W.sink_frames, W.window_frames, device=dev)
+    fill = W.held_frames + c                                 # start full: every step evicts 3 then appends 3
+    kfill = host_normal(10, (W.cache_batch, fill * T, H, D)).to(dev)
+    vfill = host_normal(11, (W.cache_batch, fill * T, H, D)).to(dev)
+    A.astro_kvcache_append(cache, kfill, vfill, fill)
+    del kfill, vfill
+    o = torch.empty_like(q); lse = torch.empty((B, H, M), dtype=torch.float32, device=dev)
+    dq = torch.empty_like(q); dk = torch.empty_like(q); dv = torch.empty_like(q)
+    delta = torch.empty((B, H, M), dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # > 126 MB L2
+    scale = W.scale
+
+    def step(ev=None):
+        """Device-resident step; `ev` collects (name, start, end) events per stage when given."""
+        def stage(name, fn):
+            if ev is None:
+                fn(); return
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record(); fn(); e.record(); ev.append((name, s, e))
+        A.astro_kvcache_evict(cache, c)
+        stage("fwd", lambda: A.astro_chunk_attn_fwd(cache, q, kc, vc, scale, o=o, lse=lse))
+        stage("delta", lambda: A.astro_chunk_attn_bwd_delta(o, do, delta=delta))
+        stage("dq", lambda: A.astro_chunk_attn_bwd_dq(cache, q, kc, vc, lse, delta, do, scale, dq=dq))
+        stage("dkv", lambda: A.astro_chunk_attn_bwd_dkv(q, kc, vc, lse, delta, do, scale, dk_chunk=dk, dv_chunk=dv))
+        stage("append", lambda: A.astro_kvcache_append(cache, kc, vc, c))
+    launches_per_step = 5
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    # ---- device-timed region: K steps, each bracketed by its own events, L2 flushed between steps
+    gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", "")
+    sampler = ClockSampler(gpu_id)
+    sampler.start()
+    time.sleep(0.12)
+    barrier()
+    t_wall0 = time.time()
+    step_events, stage_events = [], []
+    for _ in range(args.steps):
+        flush.zero_()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record(); step(stage_events); e.record()
+        step_events.append((s, e))
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    ms_step_local = float(np.mean([s.elapsed_time(e) for s, e in step_events]))
+    stage_ms = {}
+    for name, s, e in stage_events:
+        stage_ms.setdefault(name, []).append(s.elapsed_time(e))
+    stage_ms = {k: float(np.mean(v)) for k, v in stage_ms.items()}
+    A.astro_last_device_status()
+    ms_step = max_over_ranks(ms_step_local, world, dev)
+    flops_step = W.fwd_flops() + W.bwd_flops()
+    value = aggregate(flops_step, ms_step, world)
+
+    # ---- end to end: the same step through the public API with host buffers, copies inside the timed region
+    h_o = torch.empty((B, M, H, D), dtype=torch.bfloat16).pin_memory()
+    h_dq, h_dk, h_dv = (torch.empty_like(h_o).pin_memory() for _ in range(3))
+    h_lse = torch.empty((B, H, M), dtype=torch.float32).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in (h_q, h_kc, h_vc, h_do))
+    d2h = sum(t.numel() * t.element_size() for t in (h_o, h_lse, h_dq, h_dk, h_dv))
+
+    def e2e_step():
+        q.copy_(h_q, non_blocking=True); kc.copy_(h_kc, non_blocking=True)
+        vc.copy_(h_vc, non_blocking=True); do.copy_(h_do, non_blocking=True)
+        step()
+        h_o.copy_(o, non_blocking=True); h_lse.copy_(lse, non_blocking=True); h_dq.copy_(dq, non_blocking=True)
+        h_dk.copy_(dk, non_blocking=True); h_dv.copy_(dv, non_blocking=True)
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    n_e2e = max(3, min(args.steps, 50))
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record()
+    for _ in range(n_e2e):
+        e2e_step()
+    e.record()
+    barrier()
+    ms_e2e = max_over_ranks(s.elapsed_time(e) / n_e2e, world, dev)
+    e2e_value = aggregate(flops_step, ms_e2e, world)
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return 0
+
+    # ---- roofline of the dominant kernel (largest share of the step), timed live above
+    kernel_flops = {"fwd": ("chunk_attn_fwd_kernel<128>", W.fwd_flops()),
+                    "dq": ("chunk_attn_bwd_dq_kernel<128>", 6.0 * B * H * M * W.total_keys * D),
+                    "dkv": ("chunk_attn_bwd_dkv_kernel<128>", 4.0 * B * H * M * M * D)}
+    dom = max(kernel_flops, key=lambda k: stage_ms[k])
+    kname, kflops = kernel_flops[dom]
+    achieved = kflops / (stage_ms[dom] * 1e-3) / 1e12
+    peak = peaks["bf16_sustained"]
+    roofline = {"bound": "tensor", "kernel": kname, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None,
+                "peak_source": "%s bf16 sustained (kernel timed inside a long loop); burst %.1f" % (peaks["source"], peaks["bf16_burst"]),
+                "frac_of_burst": achieved / peaks["bf16_burst"], "ms_per_launch": stage_ms[dom],
+                "algorithmic_flops_per_launch": kflops}
+    per_kernel = {}
+    for k, (name, fl) in kernel_flops.items():
+        t = fl / (stage_ms[k] * 1e-3) / 1e12
+        per_kernel[k] = {"kernel": name, "ms": stage_ms[k], "tflops": t, "frac_of_sustained": t / peaks["bf16_sustained"],
+                         "frac_of_burst": t / peaks["bf16_burst"]}
+    bwd_ms = stage_ms["delta"] + stage_ms["dq"] + stage_ms["dkv"]
+    per_kernel["bwd_total"] = {"ms": bwd_ms, "tflops": W.bwd_flops() / (bwd_ms * 1e-3) / 1e12}
+    append_bytes = 2 * 2 * W.cache_batch * H * c * T * D * 2
+    per_kernel["append"] = {"kernel": "ring_copy_kernel<true>", "ms": stage_ms["append"],
+                            "gbs": append_bytes / (stage_ms["append"] * 1e-3) / 1e9,
+                            "frac_of_hbm": append_bytes / (stage_ms["append"] * 1e-3) / 1e9 / peaks["hbm"]}
+    per_kernel["delta"] = {"kernel": "bwd_delta_kernel<128>", "ms": stage_ms["delta"]}
+
+    # ---- CPU oracle on a bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_rows = 4680
+        v_cpu, dt = time_oracle(n_rows, 1)
+        cpu = {"value": v_cpu, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "seconds": dt,
+               "sample": "1 of 12 heads, all 4680 query rows x 32760 keys, fwd+bwd once, fp64 numpy"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": {"workload": WORKLOAD, "l2": "flushed between timed steps (256 MB write)",
+                                            "timing": "CUDA events per step, mean over steps, max over ranks",
+                                            "parallelism": "replicas only (no exchange step)"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e},
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "roofline": roofline,
+            "cpu_baseline": cpu, "kernels": per_kernel}
+    print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    return run_reference(args) if args.impl == "reference" else run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

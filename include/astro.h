@@ -58,7 +58,7 @@ size_t astro_kvcache_storage_bytes(const astro_kvcache_desc_t* desc);
 /* Sec. 3.2, "Rolling KV Cache with Frame Sinks": bind caller-allocated device
  * storage for the restricted context C_n (S sink frames + window of L frames),
  * so that resident KV memory is constant however long the video grows.
- * k_storage/v_storage: device, >= bytes_each each, 1024-byte aligned; the layout
+ * k_storage/v_storage: device, >= bytes_each each, 16-byte aligned; the layout
  * inside is private ([B_c, H, slot, T, D]).  The storage need not be initialised.
  * The cache starts empty.  *out receives the handle. */
 astro_status_t astro_kvcache_create(const astro_kvcache_desc_t* desc, void* k_storage, void* v_storage,
@@ -127,6 +127,23 @@ astro_status_t astro_chunk_attn_bwd(const astro_kvcache_t* cache, const void* q,
                                     int batch, int heads, int head_dim, int n_q, int n_kc, float scale,
                                     void* dq, void* dk_chunk, void* dv_chunk, void* workspace,
                                     size_t workspace_bytes, void* stream);
+
+/* The three stages of astro_chunk_attn_bwd as calls of their own (same layouts, same checks); the
+ * composite call is exactly delta, then dq, then dkv on one stream.  A caller that trains only the
+ * query side can skip the last stage.
+ *   delta: delta[b,h,i] = sum_d dO[b,i,h,d] * O[b,i,h,d], fp32 [batch, H, n_q] (device, 16-byte aligned).
+ *   dq:    dQ over ALL keys (cache + chunk) from Q, dO, LSE, delta.
+ *   dkv:   dK, dV of the chunk's own keys from Q, dO, LSE, delta (no cache involved: context is detached). */
+astro_status_t astro_chunk_attn_bwd_delta(const void* o, const void* d_o, int batch, int heads, int head_dim,
+                                          int n_q, float* delta, void* stream);
+astro_status_t astro_chunk_attn_bwd_dq(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
+                                       const void* v_chunk, const float* lse, const float* delta, const void* d_o,
+                                       int batch, int heads, int head_dim, int n_q, int n_kc, float scale,
+                                       void* dq, void* stream);
+astro_status_t astro_chunk_attn_bwd_dkv(const void* q, const void* k_chunk, const void* v_chunk, const float* lse,
+                                        const float* delta, const void* d_o, int batch, int heads, int head_dim,
+                                        int n_q, int n_kc, float scale, void* dk_chunk, void* dv_chunk,
+                                        void* stream);
 
 /* Every device-side wait in the kernels is bounded; one that runs out records a
  * code in a device status word instead of hanging.  This call synchronises the

@@ -19,6 +19,7 @@ STATUS_NAMES = {0: "ASTRO_OK", 1: "ASTRO_ERR_NULL", 2: "ASTRO_ERR_SHAPE", 3: "AS
 EXPORTED = ("astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcache_destroy", "astro_kvcache_reset",
             "astro_kvcache_append", "astro_kvcache_evict", "astro_kvcache_query", "astro_kvcache_export",
             "astro_chunk_attn_fwd", "astro_chunk_attn_bwd_workspace_bytes", "astro_chunk_attn_bwd",
+            "astro_chunk_attn_bwd_delta", "astro_chunk_attn_bwd_dq", "astro_chunk_attn_bwd_dkv",
             "astro_last_device_status", "astro_status_string")
 
 
@@ -67,6 +68,12 @@ def lib():
     L.astro_chunk_attn_bwd_workspace_bytes.argtypes = [ci, ci, ci, ci]
     L.astro_chunk_attn_bwd.restype = ci
     L.astro_chunk_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp, sz, vp]
+    L.astro_chunk_attn_bwd_delta.restype = ci
+    L.astro_chunk_attn_bwd_delta.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
+    L.astro_chunk_attn_bwd_dq.restype = ci
+    L.astro_chunk_attn_bwd_dq.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp]
+    L.astro_chunk_attn_bwd_dkv.restype = ci
+    L.astro_chunk_attn_bwd_dkv.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp]
     L.astro_last_device_status.restype = ci
     L.astro_last_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.astro_status_string.restype = C.c_char_p
@@ -224,6 +231,45 @@ def astro_chunk_attn_bwd(cache, q, k_chunk, v_chunk, o, lse, d_o, scale: float, 
                                     workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "astro_chunk_attn_bwd")
     return dq, dk_chunk, dv_chunk
+
+
+def astro_chunk_attn_bwd_delta(o, d_o, delta=None, stream=None):
+    """delta [B, H, n_q] fp32 = rowsum(dO * O)."""
+    import torch
+    B, n_q, H, D = o.shape
+    if delta is None:
+        delta = torch.empty((B, H, n_q), dtype=torch.float32, device=o.device)
+    _check(lib().astro_chunk_attn_bwd_delta(_ptr(o), _ptr(d_o), B, H, D, n_q, _ptr(delta), _stream(stream)),
+           "astro_chunk_attn_bwd_delta")
+    return delta
+
+
+def astro_chunk_attn_bwd_dq(cache, q, k_chunk, v_chunk, lse, delta, d_o, scale: float, dq=None, stream=None):
+    import torch
+    B, n_q, H, D = q.shape
+    n_kc = 0 if k_chunk is None else k_chunk.shape[1]
+    if dq is None:
+        dq = torch.empty_like(q)
+    st = lib().astro_chunk_attn_bwd_dq(None if cache is None else cache.handle, _ptr(q), _ptr(k_chunk), _ptr(v_chunk),
+                                       _ptr(lse), _ptr(delta), _ptr(d_o), B, H, D, n_q, n_kc, float(scale), _ptr(dq),
+                                       _stream(stream))
+    _check(st, "astro_chunk_attn_bwd_dq")
+    return dq
+
+
+def astro_chunk_attn_bwd_dkv(q, k_chunk, v_chunk, lse, delta, d_o, scale: float, dk_chunk=None, dv_chunk=None,
+                             stream=None):
+    import torch
+    B, n_q, H, D = q.shape
+    n_kc = k_chunk.shape[1]
+    if dk_chunk is None:
+        dk_chunk = torch.empty_like(k_chunk)
+    if dv_chunk is None:
+        dv_chunk = torch.empty_like(v_chunk)
+    st = lib().astro_chunk_attn_bwd_dkv(_ptr(q), _ptr(k_chunk), _ptr(v_chunk), _ptr(lse), _ptr(delta), _ptr(d_o), B, H,
+                                        D, n_q, n_kc, float(scale), _ptr(dk_chunk), _ptr(dv_chunk), _stream(stream))
+    _check(st, "astro_chunk_attn_bwd_dkv")
+    return dk_chunk, dv_chunk
 
 
 def astro_last_device_status() -> int:

@@ -137,6 +137,15 @@ template <typename K> astro_status_t set_smem(K kernel, int bytes) {
              : ASTRO_ERR_CUDA;
 }
 
+template <typename K> astro_status_t set_smem_once(K kernel, int bytes, bool (&done)[64]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ASTRO_ERR_CUDA;
+  if (dev >= 0 && dev < 64 && done[dev]) return ASTRO_OK;
+  astro_status_t s = set_smem(kernel, bytes);
+  if (s == ASTRO_OK && dev >= 0 && dev < 64) done[dev] = true;
+  return s;
+}
+
 astro_status_t launch_status() { return cudaGetLastError() == cudaSuccess ? ASTRO_OK : ASTRO_ERR_CUDA; }
 
 struct AttnArgs {
@@ -164,12 +173,9 @@ template <int D>
 astro_status_t launch_fwd(const AttnArgs& a, const CUtensorMap& tq, const CUtensorMap& tkc, const CUtensorMap& tvc,
                           const CUtensorMap& tkx, const CUtensorMap& tvx, const KeySegs& segs, float scale, void* o,
                           float* lse, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    astro_status_t s = set_smem(chunk_attn_fwd_kernel<D>, FwdSmem<D>::kTotal);
-    if (s != ASTRO_OK) return s;
-    attr_set = true;
-  }
+  static bool done[64];
+  astro_status_t s = set_smem_once(chunk_attn_fwd_kernel<D>, FwdSmem<D>::kTotal, done);
+  if (s != ASTRO_OK) return s;
   dim3 grid((a.n_q + kTile - 1) / kTile, a.heads, a.batch);
   chunk_attn_fwd_kernel<D><<<grid, 128, FwdSmem<D>::kTotal, st>>>(
       tq, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0,
@@ -178,34 +184,42 @@ astro_status_t launch_fwd(const AttnArgs& a, const CUtensorMap& tq, const CUtens
 }
 
 template <int D>
-astro_status_t launch_bwd(const AttnArgs& a, const CUtensorMap& tq, const CUtensorMap& tdo, const CUtensorMap& tkc,
-                          const CUtensorMap& tvc, const CUtensorMap& tkx, const CUtensorMap& tvx, const KeySegs& segs,
-                          float scale, const void* o, const float* lse, const void* d_o, float* delta, void* dq,
-                          void* dk, void* dv, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    astro_status_t s = set_smem(chunk_attn_bwd_dq_kernel<D>, BwdSmem<D>::kTotal);
-    if (s != ASTRO_OK) return s;
-    s = set_smem(chunk_attn_bwd_dkv_kernel<D>, BwdSmem<D>::kTotal);
-    if (s != ASTRO_OK) return s;
-    attr_set = true;
-  }
-  const long long rows = static_cast<long long>(a.batch) * a.n_q * a.heads;
-  const unsigned delta_blocks = static_cast<unsigned>((rows * 32 + 255) / 256);
-  bwd_delta_kernel<D><<<delta_blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(o),
-                                                   static_cast<const __nv_bfloat16*>(d_o), delta, a.batch, a.n_q,
-                                                   a.heads);
+astro_status_t launch_bwd_delta(const void* o, const void* d_o, int batch, int heads, int n_q, float* delta,
+                                cudaStream_t st) {
+  const long long rows = static_cast<long long>(batch) * n_q * heads;
+  const unsigned blocks = static_cast<unsigned>((rows * 32 + 255) / 256);
+  bwd_delta_kernel<D><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(o),
+                                             static_cast<const __nv_bfloat16*>(d_o), delta, batch, n_q, heads);
+  return launch_status();
+}
+
+template <int D>
+astro_status_t launch_bwd_dq(const AttnArgs& a, const CUtensorMap& tq, const CUtensorMap& tdo, const CUtensorMap& tkc,
+                             const CUtensorMap& tvc, const CUtensorMap& tkx, const CUtensorMap& tvx,
+                             const KeySegs& segs, float scale, const float* lse, const float* delta, void* dq,
+                             cudaStream_t st) {
+  static bool done[64];
+  astro_status_t s = set_smem_once(chunk_attn_bwd_dq_kernel<D>, BwdSmem<D>::kTotal, done);
+  if (s != ASTRO_OK) return s;
   dim3 grid_q((a.n_q + kTile - 1) / kTile, a.heads, a.batch);
   chunk_attn_bwd_dq_kernel<D><<<grid_q, 128, BwdSmem<D>::kTotal, st>>>(
       tq, tdo, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads,
       (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0, scale, lse, delta,
       static_cast<__nv_bfloat16*>(dq));
-  if (a.n_kc > 0) {
-    dim3 grid_k((a.n_kc + kTile - 1) / kTile, a.heads, a.batch);
-    chunk_attn_bwd_dkv_kernel<D><<<grid_k, 128, BwdSmem<D>::kTotal, st>>>(
-        tq, tdo, tkc, tvc, a.n_q, a.n_kc, a.heads, scale, lse, delta, static_cast<__nv_bfloat16*>(dk),
-        static_cast<__nv_bfloat16*>(dv));
-  }
+  return launch_status();
+}
+
+template <int D>
+astro_status_t launch_bwd_dkv(const AttnArgs& a, const CUtensorMap& tq, const CUtensorMap& tdo,
+                              const CUtensorMap& tkc, const CUtensorMap& tvc, float scale, const float* lse,
+                              const float* delta, void* dk, void* dv, cudaStream_t st) {
+  static bool done[64];
+  astro_status_t s = set_smem_once(chunk_attn_bwd_dkv_kernel<D>, BwdSmem<D>::kTotal, done);
+  if (s != ASTRO_OK) return s;
+  dim3 grid_k((a.n_kc + kTile - 1) / kTile, a.heads, a.batch);
+  chunk_attn_bwd_dkv_kernel<D><<<grid_k, 128, BwdSmem<D>::kTotal, st>>>(
+      tq, tdo, tkc, tvc, a.n_q, a.n_kc, a.heads, scale, lse, delta, static_cast<__nv_bfloat16*>(dk),
+      static_cast<__nv_bfloat16*>(dv));
   return launch_status();
 }
 
@@ -376,19 +390,29 @@ size_t astro_chunk_attn_bwd_workspace_bytes(int batch, int heads, int n_q, int h
   return (b + 255) & ~static_cast<size_t>(255);
 }
 
-astro_status_t astro_chunk_attn_bwd(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
-                                    const void* v_chunk, const void* o, const float* lse, const void* d_o, int batch,
-                                    int heads, int head_dim, int n_q, int n_kc, float scale, void* dq, void* dk_chunk,
-                                    void* dv_chunk, void* workspace, size_t workspace_bytes, void* stream) {
-  if (!q || !o || !lse || !d_o || !dq || !workspace) return ASTRO_ERR_NULL;
-  if (n_kc > 0 && (!k_chunk || !v_chunk || !dk_chunk || !dv_chunk)) return ASTRO_ERR_NULL;
+astro_status_t astro_chunk_attn_bwd_delta(const void* o, const void* d_o, int batch, int heads, int head_dim, int n_q,
+                                          float* delta, void* stream) {
+  if (!o || !d_o || !delta) return ASTRO_ERR_NULL;
+  if (batch < 1 || heads < 1 || n_q < 1 || (head_dim != 64 && head_dim != 128)) return ASTRO_ERR_SHAPE;
+  if (!aligned16(o) || !aligned16(d_o) || !aligned16(delta)) return ASTRO_ERR_ALIGN;
+  astro_status_t s = check_arch();
+  if (s != ASTRO_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return head_dim == 128 ? launch_bwd_delta<128>(o, d_o, batch, heads, n_q, delta, st)
+                         : launch_bwd_delta<64>(o, d_o, batch, heads, n_q, delta, st);
+}
+
+astro_status_t astro_chunk_attn_bwd_dq(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
+                                       const void* v_chunk, const float* lse, const float* delta, const void* d_o,
+                                       int batch, int heads, int head_dim, int n_q, int n_kc, float scale, void* dq,
+                                       void* stream) {
+  if (!q || !lse || !delta || !d_o || !dq) return ASTRO_ERR_NULL;
+  if (n_kc > 0 && (!k_chunk || !v_chunk)) return ASTRO_ERR_NULL;
   const AttnArgs a{cache, batch, heads, head_dim, n_q, n_kc};
   astro_status_t s = check_attn_args(a, scale);
   if (s != ASTRO_OK) return s;
-  if (workspace_bytes < astro_chunk_attn_bwd_workspace_bytes(batch, heads, n_q, head_dim)) return ASTRO_ERR_CAPACITY;
-  if (!aligned16(q) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) || !aligned16(workspace) ||
-      (reinterpret_cast<uintptr_t>(lse) & 3u) ||
-      (n_kc > 0 && (!aligned16(k_chunk) || !aligned16(v_chunk) || !aligned16(dk_chunk) || !aligned16(dv_chunk))))
+  if (!aligned16(q) || !aligned16(d_o) || !aligned16(dq) || (reinterpret_cast<uintptr_t>(lse) & 3u) ||
+      (reinterpret_cast<uintptr_t>(delta) & 3u) || (n_kc > 0 && (!aligned16(k_chunk) || !aligned16(v_chunk))))
     return ASTRO_ERR_ALIGN;
   s = check_arch();
   if (s != ASTRO_OK) return s;
@@ -409,11 +433,54 @@ astro_status_t astro_chunk_attn_bwd(const astro_kvcache_t* cache, const void* q,
   }
   const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return head_dim == 128 ? launch_bwd_dq<128>(a, tq, tdo, tkc, tvc, tkx, tvx, segs, scale, lse, delta, dq, st)
+                         : launch_bwd_dq<64>(a, tq, tdo, tkc, tvc, tkx, tvx, segs, scale, lse, delta, dq, st);
+}
+
+astro_status_t astro_chunk_attn_bwd_dkv(const void* q, const void* k_chunk, const void* v_chunk, const float* lse,
+                                        const float* delta, const void* d_o, int batch, int heads, int head_dim,
+                                        int n_q, int n_kc, float scale, void* dk_chunk, void* dv_chunk, void* stream) {
+  if (!q || !k_chunk || !v_chunk || !lse || !delta || !d_o || !dk_chunk || !dv_chunk) return ASTRO_ERR_NULL;
+  const AttnArgs a{nullptr, batch, heads, head_dim, n_q, n_kc};
+  astro_status_t s = check_attn_args(a, scale);
+  if (s != ASTRO_OK) return s;
+  if (!aligned16(q) || !aligned16(d_o) || !aligned16(k_chunk) || !aligned16(v_chunk) || !aligned16(dk_chunk) ||
+      !aligned16(dv_chunk) || (reinterpret_cast<uintptr_t>(lse) & 3u) || (reinterpret_cast<uintptr_t>(delta) & 3u))
+    return ASTRO_ERR_ALIGN;
+  s = check_arch();
+  if (s != ASTRO_OK) return s;
+  CUtensorMap tq, tdo, tkc, tvc;
+  if ((s = make_tmap_user(&tq, q, head_dim, n_q, heads, batch)) != ASTRO_OK) return s;
+  if ((s = make_tmap_user(&tdo, d_o, head_dim, n_q, heads, batch)) != ASTRO_OK) return s;
+  if ((s = make_tmap_user(&tkc, k_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
+  if ((s = make_tmap_user(&tvc, v_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return head_dim == 128 ? launch_bwd_dkv<128>(a, tq, tdo, tkc, tvc, scale, lse, delta, dk_chunk, dv_chunk, st)
+                         : launch_bwd_dkv<64>(a, tq, tdo, tkc, tvc, scale, lse, delta, dk_chunk, dv_chunk, st);
+}
+
+astro_status_t astro_chunk_attn_bwd(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
+                                    const void* v_chunk, const void* o, const float* lse, const void* d_o, int batch,
+                                    int heads, int head_dim, int n_q, int n_kc, float scale, void* dq, void* dk_chunk,
+                                    void* dv_chunk, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!q || !o || !lse || !d_o || !dq || !workspace) return ASTRO_ERR_NULL;
+  if (n_kc > 0 && (!k_chunk || !v_chunk || !dk_chunk || !dv_chunk)) return ASTRO_ERR_NULL;
+  const AttnArgs a{cache, batch, heads, head_dim, n_q, n_kc};
+  astro_status_t s = check_attn_args(a, scale);
+  if (s != ASTRO_OK) return s;
+  if (workspace_bytes < astro_chunk_attn_bwd_workspace_bytes(batch, heads, n_q, head_dim)) return ASTRO_ERR_CAPACITY;
+  if (!aligned16(q) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) || !aligned16(workspace) ||
+      (reinterpret_cast<uintptr_t>(lse) & 3u) ||
+      (n_kc > 0 && (!aligned16(k_chunk) || !aligned16(v_chunk) || !aligned16(dk_chunk) || !aligned16(dv_chunk))))
+    return ASTRO_ERR_ALIGN;
   float* delta = static_cast<float*>(workspace);
-  return head_dim == 128 ? launch_bwd<128>(a, tq, tdo, tkc, tvc, tkx, tvx, segs, scale, o, lse, d_o, delta, dq,
-                                           dk_chunk, dv_chunk, st)
-                         : launch_bwd<64>(a, tq, tdo, tkc, tvc, tkx, tvx, segs, scale, o, lse, d_o, delta, dq,
-                                          dk_chunk, dv_chunk, st);
+  s = astro_chunk_attn_bwd_delta(o, d_o, batch, heads, head_dim, n_q, delta, stream);
+  if (s != ASTRO_OK) return s;
+  s = astro_chunk_attn_bwd_dq(cache, q, k_chunk, v_chunk, lse, delta, d_o, batch, heads, head_dim, n_q, n_kc, scale,
+                              dq, stream);
+  if (s != ASTRO_OK || n_kc == 0) return s;
+  return astro_chunk_attn_bwd_dkv(q, k_chunk, v_chunk, lse, delta, d_o, batch, heads, head_dim, n_q, n_kc, scale,
+                                  dk_chunk, dv_chunk, stream);
 }
 
 astro_status_t astro_last_device_status(uint32_t* detail) {
