@@ -145,6 +145,26 @@ astro_status_t astro_chunk_attn_bwd_dkv(const void* q, const void* k_chunk, cons
                                         int n_q, int n_kc, float scale, void* dk_chunk, void* dv_chunk,
                                         void* stream);
 
+/* The paper has no counterpart for this call: it exists for callers that must not allocate device
+ * memory around the backward -- a training loop whose allocator is frozen after warm-up, a plug-in
+ * that runs inside someone else's memory pool, a host thread that may not take the allocator's lock.
+ * Such callers cannot provide the delta scratch that astro_chunk_attn_bwd asks for, so this variant
+ * keeps it in a fixed device array inside the library instead: ASTRO_BWD_STATIC_MAX_ROWS fp32 values
+ * (1 MiB), resident on every GPU that loads the library until the process exits.
+ * Same inputs, outputs, layouts and results as astro_chunk_attn_bwd, without the workspace arguments.
+ * It calls no cudaMalloc/cudaFree and no allocating library routine.
+ *   - ASTRO_ERR_CAPACITY if batch * heads * n_q exceeds ASTRO_BWD_STATIC_MAX_ROWS; nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array: two calls whose kernels may overlap on the GPU
+ *     (different streams, no ordering between them) race on it.  Calls on one stream are safe.  The
+ *     array keeps the previous call's delta; every element a call reads it has written first. */
+#define ASTRO_BWD_STATIC_MAX_ROWS 262144
+astro_status_t astro_chunk_attn_bwd_static(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
+                                           const void* v_chunk, const void* o, const float* lse, const void* d_o,
+                                           int batch, int heads, int head_dim, int n_q, int n_kc, float scale,
+                                           void* dq, void* dk_chunk, void* dv_chunk, void* stream);
+
 /* Every device-side wait in the kernels is bounded; one that runs out records a
  * code in a device status word instead of hanging.  This call synchronises the
  * current device, reads and clears that word: ASTRO_OK, or ASTRO_ERR_TIMEOUT

@@ -20,6 +20,7 @@ EXPORTED = ("astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcach
             "astro_kvcache_append", "astro_kvcache_evict", "astro_kvcache_query", "astro_kvcache_export",
             "astro_chunk_attn_fwd", "astro_chunk_attn_bwd_workspace_bytes", "astro_chunk_attn_bwd",
             "astro_chunk_attn_bwd_delta", "astro_chunk_attn_bwd_dq", "astro_chunk_attn_bwd_dkv",
+            "astro_chunk_attn_bwd_static",
             "astro_last_device_status", "astro_status_string")
 
 
@@ -74,6 +75,8 @@ def lib():
     L.astro_chunk_attn_bwd_dq.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp]
     L.astro_chunk_attn_bwd_dkv.restype = ci
     L.astro_chunk_attn_bwd_dkv.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp]
+    L.astro_chunk_attn_bwd_static.restype = ci
+    L.astro_chunk_attn_bwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
     L.astro_last_device_status.restype = ci
     L.astro_last_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.astro_status_string.restype = C.c_char_p
@@ -270,6 +273,24 @@ def astro_chunk_attn_bwd_dkv(q, k_chunk, v_chunk, lse, delta, d_o, scale: float,
                                         D, n_q, n_kc, float(scale), _ptr(dk_chunk), _ptr(dv_chunk), _stream(stream))
     _check(st, "astro_chunk_attn_bwd_dkv")
     return dk_chunk, dv_chunk
+
+
+BWD_STATIC_MAX_ROWS = 262144
+
+
+def astro_chunk_attn_bwd_static(cache, q, k_chunk, v_chunk, o, lse, d_o, scale: float, dq, dk_chunk, dv_chunk,
+                                stream=None):
+    """Backward for callers that may not allocate: no workspace argument, delta goes to a fixed 1 MiB
+    device array inside the library (batch * heads * n_q <= BWD_STATIC_MAX_ROWS).  The caller passes every
+    output tensor; this wrapper allocates nothing either.  Calls that may overlap on the GPU race on the
+    shared array; issue them on one stream."""
+    B, n_q, H, D = q.shape
+    n_kc = 0 if k_chunk is None else k_chunk.shape[1]
+    st = lib().astro_chunk_attn_bwd_static(None if cache is None else cache.handle, _ptr(q), _ptr(k_chunk),
+                                           _ptr(v_chunk), _ptr(o), _ptr(lse), _ptr(d_o), B, H, D, n_q, n_kc,
+                                           float(scale), _ptr(dq), _ptr(dk_chunk), _ptr(dv_chunk), _stream(stream))
+    _check(st, "astro_chunk_attn_bwd_static")
+    return dq, dk_chunk, dv_chunk
 
 
 def astro_last_device_status() -> int:

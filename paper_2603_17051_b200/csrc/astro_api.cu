@@ -483,6 +483,49 @@ astro_status_t astro_chunk_attn_bwd(const astro_kvcache_t* cache, const void* q,
                                   dk_chunk, dv_chunk, stream);
 }
 
+// ---- backward without caller scratch ---------------------------------------------------------------
+// delta lives in this fixed device array.  In host code `g_bwd_static_delta` is only a stand-in for the
+// symbol, not a device address: the address each GPU gives it is looked up once per device below.
+static __device__ __align__(256) float g_bwd_static_delta[ASTRO_BWD_STATIC_MAX_ROWS];
+
+static astro_status_t bwd_static_scratch(float** out) {
+  static float* addr[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ASTRO_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return ASTRO_ERR_CUDA;
+  if (!addr[dev]) {
+    float* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_bwd_static_delta) != cudaSuccess || !p)
+      return ASTRO_ERR_CUDA;
+    addr[dev] = p;
+  }
+  *out = addr[dev];
+  return ASTRO_OK;
+}
+
+astro_status_t astro_chunk_attn_bwd_static(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
+                                           const void* v_chunk, const void* o, const float* lse, const void* d_o,
+                                           int batch, int heads, int head_dim, int n_q, int n_kc, float scale,
+                                           void* dq, void* dk_chunk, void* dv_chunk, void* stream) {
+  if (!q || !o || !lse || !d_o || !dq) return ASTRO_ERR_NULL;
+  if (n_kc > 0 && (!k_chunk || !v_chunk || !dk_chunk || !dv_chunk)) return ASTRO_ERR_NULL;
+  const AttnArgs a{cache, batch, heads, head_dim, n_q, n_kc};
+  astro_status_t s = check_attn_args(a, scale);
+  if (s != ASTRO_OK) return s;
+  if (static_cast<long long>(batch) * heads * n_q > ASTRO_BWD_STATIC_MAX_ROWS) return ASTRO_ERR_CAPACITY;
+  s = check_arch();
+  if (s != ASTRO_OK) return s;
+  float* delta = nullptr;
+  if ((s = bwd_static_scratch(&delta)) != ASTRO_OK) return s;
+  s = astro_chunk_attn_bwd_delta(o, d_o, batch, heads, head_dim, n_q, delta, stream);
+  if (s != ASTRO_OK) return s;
+  s = astro_chunk_attn_bwd_dq(cache, q, k_chunk, v_chunk, lse, delta, d_o, batch, heads, head_dim, n_q, n_kc, scale,
+                              dq, stream);
+  if (s != ASTRO_OK || n_kc == 0) return s;
+  return astro_chunk_attn_bwd_dkv(q, k_chunk, v_chunk, lse, delta, d_o, batch, heads, head_dim, n_q, n_kc, scale,
+                                  dk_chunk, dv_chunk, stream);
+}
+
 astro_status_t astro_last_device_status(uint32_t* detail) {
   if (cudaDeviceSynchronize() != cudaSuccess) return ASTRO_ERR_CUDA;
   uint32_t word = 0;
