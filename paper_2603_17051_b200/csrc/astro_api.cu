@@ -177,7 +177,7 @@ astro_status_t launch_fwd(const AttnArgs& a, const CUtensorMap& tq, const CUtens
   astro_status_t s = set_smem_once(chunk_attn_fwd_kernel<D>, FwdSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
   dim3 grid((a.n_q + kTile - 1) / kTile, a.heads, a.batch);
-  chunk_attn_fwd_kernel<D><<<grid, 128, FwdSmem<D>::kTotal, st>>>(
+  chunk_attn_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kTotal, st>>>(
       tq, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0,
       scale * kLog2e, static_cast<__nv_bfloat16*>(o), lse);
   return launch_status();
