@@ -199,10 +199,10 @@ astro_status_t launch_bwd_dq(const AttnArgs& a, const CUtensorMap& tq, const CUt
                              const KeySegs& segs, float scale, const float* lse, const float* delta, void* dq,
                              cudaStream_t st) {
   static bool done[64];
-  astro_status_t s = set_smem_once(chunk_attn_bwd_dq_kernel<D>, BwdSmem<D>::kTotal, done);
+  astro_status_t s = set_smem_once(chunk_attn_bwd_dq_kernel<D>, DqSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
   dim3 grid_q((a.n_q + kTile - 1) / kTile, a.heads, a.batch);
-  chunk_attn_bwd_dq_kernel<D><<<grid_q, 128, BwdSmem<D>::kTotal, st>>>(
+  chunk_attn_bwd_dq_kernel<D><<<grid_q, kDqThreads, DqSmem<D>::kTotal, st>>>(
       tq, tdo, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads,
       (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0, scale, lse, delta,
       static_cast<__nv_bfloat16*>(dq));
@@ -214,10 +214,10 @@ astro_status_t launch_bwd_dkv(const AttnArgs& a, const CUtensorMap& tq, const CU
                               const CUtensorMap& tkc, const CUtensorMap& tvc, float scale, const float* lse,
                               const float* delta, void* dk, void* dv, cudaStream_t st) {
   static bool done[64];
-  astro_status_t s = set_smem_once(chunk_attn_bwd_dkv_kernel<D>, BwdSmem<D>::kTotal, done);
+  astro_status_t s = set_smem_once(chunk_attn_bwd_dkv_kernel<D>, DkvSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
   dim3 grid_k((a.n_kc + kTile - 1) / kTile, a.heads, a.batch);
-  chunk_attn_bwd_dkv_kernel<D><<<grid_k, 128, BwdSmem<D>::kTotal, st>>>(
+  chunk_attn_bwd_dkv_kernel<D><<<grid_k, kDkvThreads, DkvSmem<D>::kTotal, st>>>(
       tq, tdo, tkc, tvc, a.n_q, a.n_kc, a.heads, scale, lse, delta, static_cast<__nv_bfloat16*>(dk),
       static_cast<__nv_bfloat16*>(dv));
   return launch_status();

@@ -51,19 +51,28 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16* __r
   }
 }
 
-template <int D> struct BwdSmem {
-  static constexpr int kT0 = 0;                              // Q   (dQ kernel) | K (dK/dV kernel)
-  static constexpr int kT1 = TileGeom<D>::kBytes;            // dO               | V
-  static constexpr int kT2 = 2 * TileGeom<D>::kBytes;        // K tile           | Q tile
-  static constexpr int kT3 = 3 * TileGeom<D>::kBytes;        // V tile           | dO tile
-  static constexpr int kRowStats = 4 * TileGeom<D>::kBytes;  // 2 x 128 floats (dK/dV kernel)
-  static constexpr int kBars = kRowStats + 1024;
-  static constexpr int kTotal = kBars + 64 + 1024;
+// ------------------------------------------------------------------------------------------ dQ
+// Warp-specialised, one CTA (one 128-query tile) per SM:
+//   warps 0-3  group 0: keys  0..63  of every key tile      warps 4-7  group 1: keys 64..127
+//   warp  8    one thread issues every tcgen05 MMA           warp  9    one thread issues every TMA load
+// For each key tile and group g the tensor core forms S_g = Q K_g^T and dP_g = dO V_g^T (128 x 64 each);
+// the group turns them into dS_g (bf16, tensor memory) and the tensor core adds dS_g K_g into the one
+// dQ accumulator.  The MMAs of one group run while the other group does its exponentials.
+//   TMEM columns: S0 [0,64) dP0 [64,128) S1 [128,192) dP1 [192,256) dQ [256,256+D) dS0 [384,416) dS1 [416,448)
+constexpr int kDqKStages = 3, kDqVStages = 2;
+constexpr int kDqThreads = 320;
+
+template <int D> struct DqSmem {
+  static constexpr int kQ = 0;
+  static constexpr int kdO = TileGeom<D>::kBytes;
+  static constexpr int kK = 2 * TileGeom<D>::kBytes;
+  static constexpr int kV = kK + kDqKStages * TileGeom<D>::kBytes;
+  static constexpr int kBars = kV + kDqVStages * TileGeom<D>::kBytes;
+  static constexpr int kTotal = kBars + 256 + 1024;
 };
 
-// ------------------------------------------------------------------------------------------ dQ
 template <int D>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kDqThreads, 1)
 chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
                          const __grid_constant__ CUtensorMap tm_kc, const __grid_constant__ CUtensorMap tm_vc,
                          const __grid_constant__ CUtensorMap tm_kx, const __grid_constant__ CUtensorMap tm_vx,
@@ -72,31 +81,41 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                          __nv_bfloat16* __restrict__ dq) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
-  uint8_t* sQ = smem + BwdSmem<D>::kT0;
-  uint8_t* sdO = smem + BwdSmem<D>::kT1;
-  uint8_t* sK = smem + BwdSmem<D>::kT2;
-  uint8_t* sV = smem + BwdSmem<D>::kT3;
-  uint64_t* bar_q = reinterpret_cast<uint64_t*>(smem + BwdSmem<D>::kBars);
-  uint64_t* bar_kv = bar_q + 1;
-  uint64_t* bar_mma = bar_q + 2;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bar_q + 3);
+  uint8_t* sQ = smem + DqSmem<D>::kQ;
+  uint8_t* sdO = smem + DqSmem<D>::kdO;
+  uint8_t* sK = smem + DqSmem<D>::kK;
+  uint8_t* sV = smem + DqSmem<D>::kV;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + DqSmem<D>::kBars);
+  uint64_t* q_full = bars;
+  uint64_t* k_full = bars + 1;                 // [kDqKStages]
+  uint64_t* k_empty = k_full + kDqKStages;
+  uint64_t* v_full = k_empty + kDqKStages;     // [kDqVStages]
+  uint64_t* v_empty = v_full + kDqVStages;
+  uint64_t* s_full = v_empty + kDqVStages;     // [2]
+  uint64_t* ds_full = s_full + 2;              // [2]
+  uint64_t* dq_full = ds_full + 2;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(dq_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int q0 = blockIdx.x * kTile, h = blockIdx.y, b = blockIdx.z;
   const int bx = cache_shared ? 0 : b;
   constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kColS = 0, kColdP = 128, kColdQ = 256, kColdS = 384;
+  constexpr uint32_t kColS = 0, kColdP = 64 /* + 128 g */, kColdQ = 256, kColdS = 384 /* + 32 g */;
+  constexpr int kMmaWarp = 8, kTmaWarp = 9;
+  constexpr int kHalfBytes = 64 * 128;  // 64 rows of a block
 
   if (tid == 0) {
-    mbar_init(bar_q, 1);
-    mbar_init(bar_kv, 1);
-    mbar_init(bar_mma, 1);
+    mbar_init(q_full, 1);
+    for (int i = 0; i < kDqKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
+    for (int i = 0; i < kDqVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(ds_full + i, 128); }
+    mbar_init(dq_full, 1);
     *abort_flag = 0;
     fence_mbar_init();
     fence_proxy_async_smem();
   }
-  if (warp == 0) {
+  if (warp == kMmaWarp) {
     tmem_alloc(tmem_holder, kTmemCols);
     tmem_relinquish();
   }
@@ -104,92 +123,147 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
-  const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+  const int n_tiles = seg_tiles(segs);
 
-  if (tid == 0) {
-    mbar_arrive_expect_tx(bar_q, 2 * TileGeom<D>::kBytes);
-    tma_load_tile<D>(sQ, &tm_q, bar_q, q0, h, b);
-    tma_load_tile<D>(sdO, &tm_do, bar_q, q0, h, b);
-  }
-  const int row = q0 + tid;
-  const bool in_range = row < n_q;
-  const size_t stat_idx = (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0);
-  const float lse2 = in_range ? lse[stat_idx] * kLog2e : 0.f;
-  const float delta_r = in_range ? delta[stat_idx] : 0.f;
-  const float scale_log2 = scale * kLog2e;
-
-  uint32_t ph_kv = 0, ph_mma = 0;
-  bool first = true;
-  for (KeyTileIter it; !it.done(segs); it.next(segs)) {
-    const int valid = it.valid(segs);
-    if (tid == 0) {
-      mbar_arrive_expect_tx(bar_kv, 2 * TileGeom<D>::kBytes);
-      const bool fc = it.from_chunk(segs);
-      tma_load_tile<D>(sK, fc ? &tm_kc : &tm_kx, bar_kv, it.row0(segs), h, fc ? b : bx);
-      tma_load_tile<D>(sV, fc ? &tm_vc : &tm_vx, bar_kv, it.row0(segs), h, fc ? b : bx);
+  if (warp == kTmaWarp) {
+    if (lane == 0) {
+      mbar_arrive_expect_tx(q_full, 2 * TileGeom<D>::kBytes);
+      tma_load_tile<D>(sQ, &tm_q, q_full, q0, h, b);
+      tma_load_tile<D>(sdO, &tm_do, q_full, q0, h, b);
+      int j = 0;
+      for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
+        const int sk = j % kDqKStages, sv = j % kDqVStages;
+        const bool fc = it.from_chunk(segs);
+        mbar_wait_spin(k_empty + sk, ((j / kDqKStages) & 1) ^ 1, abort_flag);
+        mbar_arrive_expect_tx(k_full + sk, TileGeom<D>::kBytes);
+        tma_load_tile<D>(sK + sk * TileGeom<D>::kBytes, fc ? &tm_kc : &tm_kx, k_full + sk, it.row0(segs), h,
+                         fc ? b : bx);
+        mbar_wait_spin(v_empty + sv, ((j / kDqVStages) & 1) ^ 1, abort_flag);
+        mbar_arrive_expect_tx(v_full + sv, TileGeom<D>::kBytes);
+        tma_load_tile<D>(sV + sv * TileGeom<D>::kBytes, fc ? &tm_vc : &tm_vx, v_full + sv, it.row0(segs), h,
+                         fc ? b : bx);
+      }
     }
-    if (first) mbar_wait(bar_q, 0, abort_flag);
-    mbar_wait(bar_kv, ph_kv, abort_flag);
-    ph_kv ^= 1;
-    if (valid < kTile) zero_tile_rows_from<D>(sK, valid, tid);  // dS is 0 there, but 0 * NaN is NaN
-    __syncthreads();
-
-    if (tid == 0) {
+  } else if (warp == kMmaWarp) {
+    if (lane == 0) {
+      // S_g and dP_g of tile j for group g; both buffers are free once the group has published dS_g(j-1)
+      auto issue_sdp = [&](int j, int g) {
+        const uint32_t kt = smem_u32(sK + (j % kDqKStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
+        const uint32_t vt = smem_u32(sV + (j % kDqVStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
+        mma_abT<D, 64>(tmem_base + kColS + g * 128, smem_u32(sQ), kt);
+        mma_abT<D, 64>(tmem_base + kColdP + g * 128, smem_u32(sdO), vt);
+        mma_commit(s_full + g);
+      };
+      auto wait_kv = [&](int j) {
+        mbar_wait_spin(k_full + j % kDqKStages, (j / kDqKStages) & 1, abort_flag);
+        mbar_wait_spin(v_full + j % kDqVStages, (j / kDqVStages) & 1, abort_flag);
+        tc_fence_after_sync();
+      };
+      auto issue_dq = [&](int j, int g) {
+        mbar_wait_spin(ds_full + g, j & 1, abort_flag);
+        tc_fence_after_sync();
+        const uint32_t kt = smem_u32(sK + (j % kDqKStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
+        mma_pb<D, 64>(tmem_base + kColdQ, tmem_base + kColdS + g * 32, kt, j > 0 || g > 0);
+      };
+      mbar_wait_spin(q_full, 0, abort_flag);
+      wait_kv(0);
+      issue_sdp(0, 0);
+      issue_sdp(0, 1);
+      mma_commit(v_empty + 0);
+      for (int j = 0; j < n_tiles; ++j) {
+        issue_dq(j, 0);
+        if (j + 1 < n_tiles) {
+          wait_kv(j + 1);
+          issue_sdp(j + 1, 0);
+        }
+        issue_dq(j, 1);
+        mma_commit(k_empty + j % kDqKStages);
+        if (j + 1 < n_tiles) {
+          issue_sdp(j + 1, 1);
+          mma_commit(v_empty + (j + 1) % kDqVStages);
+        }
+      }
+      mma_commit(dq_full);
+    }
+  } else {
+    const int g = warp >> 2;
+    const int r = tid & 127;
+    const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const int row = q0 + r;
+    const bool in_range = row < n_q;
+    const size_t stat_idx = (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0);
+    const float lse2 = in_range ? lse[stat_idx] * kLog2e : 0.f;
+    const float delta_r = in_range ? delta[stat_idx] : 0.f;
+    const float scale_log2 = scale * kLog2e;
+    int j = 0;
+    for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
+      const int valid = it.valid(segs) - 64 * g;  // valid keys of this group's half (may be <= 0)
+      mbar_wait(s_full + g, j & 1, abort_flag);
       tc_fence_after_sync();
-      mma_abT<D>(tmem_base + kColS, smem_u32(sQ), smem_u32(sK));
-      mma_abT<D>(tmem_base + kColdP, smem_u32(sdO), smem_u32(sV));
-      mma_commit(bar_mma);
-    }
-    mbar_wait(bar_mma, ph_mma, abort_flag);
-    ph_mma ^= 1;
-    tc_fence_after_sync();
-
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t s[32], dp[32], ds[16];
-      tmem_ld32(tmem_lane + kColS + j * 32, s);
-      tmem_ld32(tmem_lane + kColdP + j * 32, dp);
+      uint32_t s[2][32], dp[2][32], ds[32];
+      tmem_ld32(tmem_lane + kColS + g * 128, s[0]);
+      tmem_ld32(tmem_lane + kColS + g * 128 + 32, s[1]);
+      tmem_ld32(tmem_lane + kColdP + g * 128, dp[0]);
+      tmem_ld32(tmem_lane + kColdP + g * 128 + 32, dp[1]);
       tmem_wait_ld();
 #pragma unroll
-      for (int c = 0; c < 32; c += 2) {
-        const float p0 = fast_exp2(fmaf(__uint_as_float(s[c]), scale_log2, -lse2));
-        const float p1 = fast_exp2(fmaf(__uint_as_float(s[c + 1]), scale_log2, -lse2));
-        float d0 = p0 * (__uint_as_float(dp[c]) - delta_r);
-        float d1 = p1 * (__uint_as_float(dp[c + 1]) - delta_r);
-        if (valid < kTile) {
-          if (j * 32 + c >= valid) d0 = 0.f;
-          if (j * 32 + c + 1 >= valid) d1 = 0.f;
+      for (int c2 = 0; c2 < 2; ++c2)
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(s[c2][c]), scale_log2, -lse2));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(s[c2][c + 1]), scale_log2, -lse2));
+          float d0 = p0 * (__uint_as_float(dp[c2][c]) - delta_r);
+          float d1 = p1 * (__uint_as_float(dp[c2][c + 1]) - delta_r);
+          if (valid < 64) {
+            if (c2 * 32 + c >= valid) d0 = 0.f;
+            if (c2 * 32 + c + 1 >= valid) d1 = 0.f;
+          }
+          ds[c2 * 16 + (c >> 1)] = pack_bf16(d0, d1);
         }
-        ds[c >> 1] = pack_bf16(d0, d1);
-      }
-      tmem_st16(tmem_lane + kColdS + j * 16, ds);
+      tmem_st32(tmem_lane + kColdS + g * 32, ds);
+      // Key rows past the segment's end may hold stale cache contents: dS is 0 there, but 0 * NaN is NaN.
+      // Group 0 clears them (all 128 rows' worth) before it publishes dS_0, which both dQ MMAs wait for.
+      if (g == 0 && it.valid(segs) < kTile)
+        zero_tile_rows_from<D>(sK + (j % kDqKStages) * TileGeom<D>::kBytes, it.valid(segs), r);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(ds_full + g);
     }
-    tmem_wait_st();
-    tc_fence_before_sync();
-    __syncthreads();
-
-    if (tid == 0) {
-      tc_fence_after_sync();
-      mma_pb<D>(tmem_base + kColdQ, tmem_base + kColdS, smem_u32(sK), !first);
-      mma_commit(bar_mma);
-    }
-    mbar_wait(bar_mma, ph_mma, abort_flag);
-    ph_mma ^= 1;
+    // ---- epilogue: group g writes columns [g D/2, (g+1) D/2) of dQ
+    mbar_wait(dq_full, 0, abort_flag);
     tc_fence_after_sync();
-    first = false;
+    __nv_bfloat16* dst = dq + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + g * (D / 2);
+    store_row_from_tmem<D / 2>(tmem_lane + kColdQ + g * (D / 2), scale, dst, in_range);
   }
-
-  const size_t row_off = ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D;
-  store_row_from_tmem<D>(tmem_lane + kColdQ, scale, dq + row_off, in_range);
 
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------------------ dK, dV
+// Warp-specialised, one CTA (one 128-key tile of the chunk) per SM; K and V of the tile stay in shared
+// memory and the query tiles stream through a 2-deep ring of (Q, dO) pairs:
+//   warps 0-3  group 0: queries  0..63 of every query tile    warps 4-7  group 1: queries 64..127
+//   warp  8    MMA issuer                                       warp  9    TMA producer
+// Per query tile and group g: S^T_g = K Q_g^T and dP^T_g = V dO_g^T (128 keys x 64 queries; one key row per
+// thread), P^T_g and dS^T_g are written over them as bf16, then dV += P^T_g dO_g and dK += dS^T_g Q_g.
+//   TMEM columns: S^T0 [0,64) dP^T0 [64,128) S^T1 [128,192) dP^T1 [192,256) dK [256,256+D) dV [384,384+D)
+constexpr int kDkvStages = 2;
+constexpr int kDkvThreads = 320;
+
+template <int D> struct DkvSmem {
+  static constexpr int kK = 0;
+  static constexpr int kV = TileGeom<D>::kBytes;
+  static constexpr int kQ = 2 * TileGeom<D>::kBytes;                      // [kDkvStages]
+  static constexpr int kdO = kQ + kDkvStages * TileGeom<D>::kBytes;       // [kDkvStages]
+  static constexpr int kStats = kdO + kDkvStages * TileGeom<D>::kBytes;   // float2 [2][128]: (lse*log2e, delta)
+  static constexpr int kBars = kStats + 2 * kTile * 8;
+  static constexpr int kTotal = kBars + 256 + 1024;
+};
+
 template <int D>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(kDkvThreads, 1)
 chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
                           const __grid_constant__ CUtensorMap tm_kc, const __grid_constant__ CUtensorMap tm_vc,
                           const int n_q, const int n_kc, const int heads, const float scale,
@@ -197,33 +271,39 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                           __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
-  uint8_t* sK = smem + BwdSmem<D>::kT0;
-  uint8_t* sV = smem + BwdSmem<D>::kT1;
-  uint8_t* sQ = smem + BwdSmem<D>::kT2;
-  uint8_t* sdO = smem + BwdSmem<D>::kT3;
-  float* sLse2 = reinterpret_cast<float*>(smem + BwdSmem<D>::kRowStats);
-  float* sDelta = sLse2 + kTile;
-  uint64_t* bar_kv = reinterpret_cast<uint64_t*>(smem + BwdSmem<D>::kBars);
-  uint64_t* bar_q = bar_kv + 1;
-  uint64_t* bar_mma = bar_kv + 2;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bar_kv + 3);
+  uint8_t* sK = smem + DkvSmem<D>::kK;
+  uint8_t* sV = smem + DkvSmem<D>::kV;
+  uint8_t* sQ = smem + DkvSmem<D>::kQ;
+  uint8_t* sdO = smem + DkvSmem<D>::kdO;
+  float2* sStat = reinterpret_cast<float2*>(smem + DkvSmem<D>::kStats);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + DkvSmem<D>::kBars);
+  uint64_t* kv_full = bars;
+  uint64_t* q_full = bars + 1;                 // [kDkvStages]
+  uint64_t* q_empty = q_full + kDkvStages;
+  uint64_t* s_full = q_empty + kDkvStages;     // [2]
+  uint64_t* p_full = s_full + 2;               // [2]
+  uint64_t* acc_full = p_full + 2;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int k0 = blockIdx.x * kTile, h = blockIdx.y, b = blockIdx.z;
   constexpr uint32_t kTmemCols = 512;
-  // P^T overlays S^T and dS^T overlays dP^T: a thread rewrites only columns it has already read.
-  constexpr uint32_t kColSt = 0, kColPt = 0, kColdPt = 128, kColdSt = 128, kColdK = 256, kColdV = 384;
+  constexpr uint32_t kColSt = 0, kColdPt = 64 /* + 128 g */, kColdK = 256, kColdV = 384;
+  constexpr int kMmaWarp = 8, kTmaWarp = 9;
+  constexpr int kHalfBytes = 64 * 128;
+  const int n_tiles = (n_q + kTile - 1) / kTile;
 
   if (tid == 0) {
-    mbar_init(bar_kv, 1);
-    mbar_init(bar_q, 1);
-    mbar_init(bar_mma, 1);
+    mbar_init(kv_full, 1);
+    for (int i = 0; i < kDkvStages; ++i) { mbar_init(q_full + i, 1); mbar_init(q_empty + i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); }
+    mbar_init(acc_full, 1);
     *abort_flag = 0;
     fence_mbar_init();
     fence_proxy_async_smem();
   }
-  if (warp == 0) {
+  if (warp == kMmaWarp) {
     tmem_alloc(tmem_holder, kTmemCols);
     tmem_relinquish();
   }
@@ -231,90 +311,111 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
-  const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
 
-  if (tid == 0) {
-    mbar_arrive_expect_tx(bar_kv, 2 * TileGeom<D>::kBytes);
-    tma_load_tile<D>(sK, &tm_kc, bar_kv, k0, h, b);
-    tma_load_tile<D>(sV, &tm_vc, bar_kv, k0, h, b);
-  }
-  const float scale_log2 = scale * kLog2e;
-  const size_t stat_base = (static_cast<size_t>(b) * heads + h) * n_q;
-
-  uint32_t ph_q = 0, ph_mma = 0;
-  bool first = true;
-  for (int q0 = 0; q0 < n_q; q0 += kTile) {
-    const int valid = min(kTile, n_q - q0);
-    if (tid == 0) {
-      mbar_arrive_expect_tx(bar_q, 2 * TileGeom<D>::kBytes);
-      tma_load_tile<D>(sQ, &tm_q, bar_q, q0, h, b);
-      tma_load_tile<D>(sdO, &tm_do, bar_q, q0, h, b);
+  if (warp == kTmaWarp) {
+    if (lane == 0) {
+      mbar_arrive_expect_tx(kv_full, 2 * TileGeom<D>::kBytes);
+      tma_load_tile<D>(sK, &tm_kc, kv_full, k0, h, b);
+      tma_load_tile<D>(sV, &tm_vc, kv_full, k0, h, b);
+      for (int i = 0; i < n_tiles; ++i) {
+        const int st = i % kDkvStages;
+        mbar_wait_spin(q_empty + st, ((i / kDkvStages) & 1) ^ 1, abort_flag);
+        mbar_arrive_expect_tx(q_full + st, 2 * TileGeom<D>::kBytes);
+        tma_load_tile<D>(sQ + st * TileGeom<D>::kBytes, &tm_q, q_full + st, i * kTile, h, b);
+        tma_load_tile<D>(sdO + st * TileGeom<D>::kBytes, &tm_do, q_full + st, i * kTile, h, b);
+      }
     }
-    sLse2[tid] = (tid < valid) ? lse[stat_base + q0 + tid] * kLog2e : 0.f;
-    sDelta[tid] = (tid < valid) ? delta[stat_base + q0 + tid] : 0.f;
-    if (first) mbar_wait(bar_kv, 0, abort_flag);
-    mbar_wait(bar_q, ph_q, abort_flag);
-    ph_q ^= 1;
-    __syncthreads();
-
-    if (tid == 0) {
+  } else if (warp == kMmaWarp) {
+    if (lane == 0) {
+      auto issue_sdp = [&](int i, int g) {
+        const uint32_t qt = smem_u32(sQ + (i % kDkvStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
+        const uint32_t dot = smem_u32(sdO + (i % kDkvStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
+        mma_abT<D, 64>(tmem_base + kColSt + g * 128, smem_u32(sK), qt);
+        mma_abT<D, 64>(tmem_base + kColdPt + g * 128, smem_u32(sV), dot);
+        mma_commit(s_full + g);
+      };
+      auto issue_acc = [&](int i, int g) {
+        mbar_wait_spin(p_full + g, i & 1, abort_flag);
+        tc_fence_after_sync();
+        const uint32_t qt = smem_u32(sQ + (i % kDkvStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
+        const uint32_t dot = smem_u32(sdO + (i % kDkvStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
+        mma_pb<D, 64>(tmem_base + kColdV, tmem_base + kColSt + g * 128, dot, i > 0 || g > 0);
+        mma_pb<D, 64>(tmem_base + kColdK, tmem_base + kColdPt + g * 128, qt, i > 0 || g > 0);
+      };
+      auto wait_q = [&](int i) {
+        mbar_wait_spin(q_full + i % kDkvStages, (i / kDkvStages) & 1, abort_flag);
+        tc_fence_after_sync();
+      };
+      mbar_wait_spin(kv_full, 0, abort_flag);
+      wait_q(0);
+      issue_sdp(0, 0);
+      issue_sdp(0, 1);
+      for (int i = 0; i < n_tiles; ++i) {
+        issue_acc(i, 0);
+        if (i + 1 < n_tiles) {
+          wait_q(i + 1);
+          issue_sdp(i + 1, 0);
+        }
+        issue_acc(i, 1);
+        mma_commit(q_empty + i % kDkvStages);
+        if (i + 1 < n_tiles) issue_sdp(i + 1, 1);
+      }
+      mma_commit(acc_full);
+    }
+  } else {
+    const int g = warp >> 2;
+    const int r = tid & 127;  // key row inside the tile = TMEM lane
+    const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+    const float scale_log2 = scale * kLog2e;
+    const size_t stat_base = (static_cast<size_t>(b) * heads + h) * n_q;
+    for (int i = 0; i < n_tiles; ++i) {
+      // per-query constants of this group's 64 queries; +inf as LSE turns rows past n_q into P = 0
+      float2* stat = sStat + (i & 1) * kTile + g * 64;
+      if (r < 64) {
+        const int qi = i * kTile + g * 64 + r;
+        stat[r] = qi < n_q ? make_float2(lse[stat_base + qi] * kLog2e, delta[stat_base + qi])
+                           : make_float2(INFINITY, 0.f);
+      }
+      named_barrier_sync(1 + g, 128);
+      mbar_wait(s_full + g, i & 1, abort_flag);
       tc_fence_after_sync();
-      mma_abT<D>(tmem_base + kColSt, smem_u32(sK), smem_u32(sQ));
-      mma_abT<D>(tmem_base + kColdPt, smem_u32(sV), smem_u32(sdO));
-      mma_commit(bar_mma);
-    }
-    mbar_wait(bar_mma, ph_mma, abort_flag);
-    ph_mma ^= 1;
-    tc_fence_after_sync();
-
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      uint32_t s[32], dp[32], pt[16], ds[16];
-      tmem_ld32(tmem_lane + kColSt + j * 32, s);
-      tmem_ld32(tmem_lane + kColdPt + j * 32, dp);
+      uint32_t s[2][32], dp[2][32], pt[32], ds[32];
+      tmem_ld32(tmem_lane + kColSt + g * 128, s[0]);
+      tmem_ld32(tmem_lane + kColSt + g * 128 + 32, s[1]);
+      tmem_ld32(tmem_lane + kColdPt + g * 128, dp[0]);
+      tmem_ld32(tmem_lane + kColdPt + g * 128 + 32, dp[1]);
       tmem_wait_ld();
 #pragma unroll
-      for (int c = 0; c < 32; c += 2) {
-        const int qa = j * 32 + c;
-        float p0 = fast_exp2(fmaf(__uint_as_float(s[c]), scale_log2, -sLse2[qa]));
-        float p1 = fast_exp2(fmaf(__uint_as_float(s[c + 1]), scale_log2, -sLse2[qa + 1]));
-        if (valid < kTile) {  // query rows past n_q: zero Q and dO rows, no LSE
-          if (qa >= valid) p0 = 0.f;
-          if (qa + 1 >= valid) p1 = 0.f;
+      for (int c2 = 0; c2 < 2; ++c2)
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const float4 st2 = *reinterpret_cast<const float4*>(stat + c2 * 32 + c);  // (lse2, delta) x 2 queries
+          const float p0 = fast_exp2(fmaf(__uint_as_float(s[c2][c]), scale_log2, -st2.x));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(s[c2][c + 1]), scale_log2, -st2.z));
+          const float d0 = p0 * (__uint_as_float(dp[c2][c]) - st2.y);
+          const float d1 = p1 * (__uint_as_float(dp[c2][c + 1]) - st2.w);
+          pt[c2 * 16 + (c >> 1)] = pack_bf16(p0, p1);
+          ds[c2 * 16 + (c >> 1)] = pack_bf16(d0, d1);
         }
-        const float d0 = p0 * (__uint_as_float(dp[c]) - sDelta[qa]);
-        const float d1 = p1 * (__uint_as_float(dp[c + 1]) - sDelta[qa + 1]);
-        pt[c >> 1] = pack_bf16(p0, p1);
-        ds[c >> 1] = pack_bf16(d0, d1);
-      }
-      tmem_st16(tmem_lane + kColPt + j * 16, pt);
-      tmem_st16(tmem_lane + kColdSt + j * 16, ds);
+      // in place: every column of S^T_g and dP^T_g this thread owns is already in registers
+      tmem_st32(tmem_lane + kColSt + g * 128, pt);
+      tmem_st32(tmem_lane + kColdPt + g * 128, ds);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(p_full + g);
     }
-    tmem_wait_st();
-    tc_fence_before_sync();
-    __syncthreads();
-
-    if (tid == 0) {
-      tc_fence_after_sync();
-      mma_pb<D>(tmem_base + kColdV, tmem_base + kColPt, smem_u32(sdO), !first);
-      mma_pb<D>(tmem_base + kColdK, tmem_base + kColdSt, smem_u32(sQ), !first);
-      mma_commit(bar_mma);
-    }
-    mbar_wait(bar_mma, ph_mma, abort_flag);
-    ph_mma ^= 1;
+    mbar_wait(acc_full, 0, abort_flag);
     tc_fence_after_sync();
-    first = false;
+    const int krow = k0 + r;
+    const bool in_range = krow < n_kc;
+    const size_t row_off = ((static_cast<size_t>(b) * n_kc + (in_range ? krow : 0)) * heads + h) * D + g * (D / 2);
+    store_row_from_tmem<D / 2>(tmem_lane + kColdK + g * (D / 2), scale, dk + row_off, in_range);
+    store_row_from_tmem<D / 2>(tmem_lane + kColdV + g * (D / 2), 1.f, dv + row_off, in_range);
   }
-
-  const int krow = k0 + tid;
-  const bool in_range = krow < n_kc;
-  const size_t row_off = ((static_cast<size_t>(b) * n_kc + (in_range ? krow : 0)) * heads + h) * D;
-  store_row_from_tmem<D>(tmem_lane + kColdK, scale, dk + row_off, in_range);
-  store_row_from_tmem<D>(tmem_lane + kColdV, 1.f, dv + row_off, in_range);
 
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 }  // namespace astro

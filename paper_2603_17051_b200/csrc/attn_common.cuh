@@ -52,10 +52,11 @@ __device__ __forceinline__ void tma_load_tile(uint8_t* smem_tile, const CUtensor
     tma_load_4d(smem_tile + blk * TileGeom<D>::kBlockBytes, tm, bar, blk * 64, row0, h, b);
 }
 
-// acc[128 x 128] = A[128 x D] * B[128 x D]^T, both tiles K-major (contraction over D).
-template <int D>
+// acc[128 x N] = A[128 x D] * B[N x D]^T, both tiles K-major (contraction over D).  B may start at any
+// multiple of 8 rows inside a 128-row tile (b_smem + rows * 128).
+template <int D, int N = kTile>
 __device__ __forceinline__ void mma_abT(uint32_t d_tmem, uint32_t a_smem, uint32_t b_smem) {
-  constexpr uint32_t idesc = make_idesc_bf16(kTile, kTile, false, false);
+  constexpr uint32_t idesc = make_idesc_bf16(kTile, N, false, false);
 #pragma unroll
   for (int k = 0; k < D / 16; ++k) {
     const uint32_t off = (k >> 2) * TileGeom<D>::kBlockBytes + (k & 3) * 32;
@@ -63,12 +64,13 @@ __device__ __forceinline__ void mma_abT(uint32_t d_tmem, uint32_t a_smem, uint32
   }
 }
 
-// acc[128 x D] (+)= A_tmem[128 x 128 bf16] * B[128 x D] with the contraction over B's rows (MN-major B).
-template <int D>
+// acc[128 x D] (+)= A_tmem[128 x KROWS bf16] * B[KROWS x D] with the contraction over B's rows (MN-major
+// B); B starts at row (b_smem - tile base) / 128 of a 128-row tile, a multiple of 16.
+template <int D, int KROWS = kTile>
 __device__ __forceinline__ void mma_pb(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_smem, bool accumulate) {
   constexpr uint32_t idesc = make_idesc_bf16(kTile, D, false, true);
 #pragma unroll
-  for (int k = 0; k < kTile / 16; ++k)
+  for (int k = 0; k < KROWS / 16; ++k)
     mma_ts(d_tmem, a_tmem + k * 8, desc_mnmajor(b_smem + k * 2048, TileGeom<D>::kBlockBytes), idesc,
            (accumulate || k > 0) ? 1u : 0u);
 }

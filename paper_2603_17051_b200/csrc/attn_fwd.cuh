@@ -26,10 +26,6 @@ template <int D> struct FwdSmem {
 
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: stale row max tolerated before O is rescaled
 
-__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 chunk_attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,

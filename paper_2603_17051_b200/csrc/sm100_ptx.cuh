@@ -80,6 +80,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return ok;
 }
 
+// Barrier among `threads` threads of the CTA (a multiple of 32) that all name the same id (1..15).
+__device__ __forceinline__ void named_barrier_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // ---------------------------------------------------------------- TMA (tiled, 4-D, no multicast)
 // Coordinates are {d, token, head, batch}; the innermost one must be a multiple of 8 bf16.
 __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* tmap, uint64_t* bar, int c0,
