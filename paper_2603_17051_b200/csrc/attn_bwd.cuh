@@ -53,14 +53,17 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16* __r
 
 // ------------------------------------------------------------------------------------------ dQ
 // Warp-specialised, one CTA (one 128-query tile) per SM:
-//   warps 0-3  group 0: keys  0..63  of every key tile      warps 4-7  group 1: keys 64..127
+//   warps 0-3  group 0: keys  0..63  of every key tile (one query row per thread)
+//   warps 4-7  group 1: keys 64..127
 //   warp  8    one thread issues every tcgen05 MMA           warp  9    one thread issues every TMA load
-// For each key tile and group g the tensor core forms S_g = Q K_g^T and dP_g = dO V_g^T (128 x 64 each);
-// the group turns them into dS_g (bf16, tensor memory) and the tensor core adds dS_g K_g into the one
-// dQ accumulator.  The MMAs of one group run while the other group does its exponentials.
-//   TMEM columns: S0 [0,64) dP0 [64,128) S1 [128,192) dP1 [192,256) dQ [256,256+D) dS0 [384,416) dS1 [416,448)
+// Per key tile j the tensor core forms S(j) = Q K^T (two tiles ahead, two buffers) and dP(j) = dO V^T (one
+// buffer), both full 128x128 MMAs.  Each thread exponentiates its 64 S values while the tensor core is busy
+// with the previous tile's dQ and this tile's dP, then turns dP into dS = P o (dP - delta) in place (bf16
+// pairs over its own dP columns) and the tensor core adds dS K into the one dQ accumulator.
+//   TMEM columns: S buffer 0 [0,128)  S buffer 1 [128,256)  dP / dS [256,384)  dQ [384,384+D)
 constexpr int kDqKStages = 3, kDqVStages = 2;
 constexpr int kDqThreads = 320;
+constexpr int kDqPolyOf8 = 2;  // share of the exponentials evaluated on the FMA pipe
 
 template <int D> struct DqSmem {
   static constexpr int kQ = 0;
@@ -91,9 +94,10 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   uint64_t* k_empty = k_full + kDqKStages;
   uint64_t* v_full = k_empty + kDqKStages;     // [kDqVStages]
   uint64_t* v_empty = v_full + kDqVStages;
-  uint64_t* s_full = v_empty + kDqVStages;     // [2]
-  uint64_t* ds_full = s_full + 2;              // [2]
-  uint64_t* dq_full = ds_full + 2;
+  uint64_t* s_full = v_empty + kDqVStages;     // [2] per S buffer
+  uint64_t* dp_full = s_full + 2;
+  uint64_t* ds_full = dp_full + 1;             // 256 arrivals: both groups
+  uint64_t* dq_full = ds_full + 1;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(dq_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
@@ -101,15 +105,19 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   const int q0 = blockIdx.x * kTile, h = blockIdx.y, b = blockIdx.z;
   const int bx = cache_shared ? 0 : b;
   constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kColS = 0, kColdP = 64 /* + 128 g */, kColdQ = 256, kColdS = 384 /* + 32 g */;
+  constexpr uint32_t kColS = 0 /* + 128 * buffer */, kColdP = 256, kColdQ = 384;
   constexpr int kMmaWarp = 8, kTmaWarp = 9;
   constexpr int kHalfBytes = 64 * 128;  // 64 rows of a block
+  const int n_tiles = seg_tiles(segs);
 
   if (tid == 0) {
     mbar_init(q_full, 1);
     for (int i = 0; i < kDqKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
     for (int i = 0; i < kDqVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(ds_full + i, 128); }
+    mbar_init(s_full, 1);
+    mbar_init(s_full + 1, 1);
+    mbar_init(dp_full, 1);
+    mbar_init(ds_full, 256);
     mbar_init(dq_full, 1);
     *abort_flag = 0;
     fence_mbar_init();
@@ -123,65 +131,70 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_holder;
-  const int n_tiles = seg_tiles(segs);
 
   if (warp == kTmaWarp) {
     if (lane == 0) {
       mbar_arrive_expect_tx(q_full, 2 * TileGeom<D>::kBytes);
       tma_load_tile<D>(sQ, &tm_q, q_full, q0, h, b);
       tma_load_tile<D>(sdO, &tm_do, q_full, q0, h, b);
-      int j = 0;
-      for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
-        const int sk = j % kDqKStages, sv = j % kDqVStages;
-        const bool fc = it.from_chunk(segs);
-        mbar_wait_spin(k_empty + sk, ((j / kDqKStages) & 1) ^ 1, abort_flag);
-        mbar_arrive_expect_tx(k_full + sk, TileGeom<D>::kBytes);
-        tma_load_tile<D>(sK + sk * TileGeom<D>::kBytes, fc ? &tm_kc : &tm_kx, k_full + sk, it.row0(segs), h,
+      // K runs one tile ahead of V: K0 K1 | V0 K2 | V1 K3 | ...  (S is issued two tiles ahead, dP one)
+      KeyTileIter itk, itv;
+      auto load_k = [&](int j) {
+        const int st = j % kDqKStages;
+        const bool fc = itk.from_chunk(segs);
+        mbar_wait_spin(k_empty + st, ((j / kDqKStages) & 1) ^ 1, abort_flag);
+        mbar_arrive_expect_tx(k_full + st, TileGeom<D>::kBytes);
+        tma_load_tile<D>(sK + st * TileGeom<D>::kBytes, fc ? &tm_kc : &tm_kx, k_full + st, itk.row0(segs), h,
                          fc ? b : bx);
-        mbar_wait_spin(v_empty + sv, ((j / kDqVStages) & 1) ^ 1, abort_flag);
-        mbar_arrive_expect_tx(v_full + sv, TileGeom<D>::kBytes);
-        tma_load_tile<D>(sV + sv * TileGeom<D>::kBytes, fc ? &tm_vc : &tm_vx, v_full + sv, it.row0(segs), h,
+        itk.next(segs);
+      };
+      auto load_v = [&](int j) {
+        const int st = j % kDqVStages;
+        const bool fc = itv.from_chunk(segs);
+        mbar_wait_spin(v_empty + st, ((j / kDqVStages) & 1) ^ 1, abort_flag);
+        mbar_arrive_expect_tx(v_full + st, TileGeom<D>::kBytes);
+        tma_load_tile<D>(sV + st * TileGeom<D>::kBytes, fc ? &tm_vc : &tm_vx, v_full + st, itv.row0(segs), h,
                          fc ? b : bx);
+        itv.next(segs);
+      };
+      load_k(0);
+      if (n_tiles > 1) load_k(1);
+      for (int j = 0; j < n_tiles; ++j) {
+        load_v(j);
+        if (j + 2 < n_tiles) load_k(j + 2);
       }
     }
   } else if (warp == kMmaWarp) {
     if (lane == 0) {
-      // S_g and dP_g of tile j for group g; both buffers are free once the group has published dS_g(j-1)
-      auto issue_sdp = [&](int j, int g) {
-        const uint32_t kt = smem_u32(sK + (j % kDqKStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
-        const uint32_t vt = smem_u32(sV + (j % kDqVStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
-        mma_abT<D, 64>(tmem_base + kColS + g * 128, smem_u32(sQ), kt);
-        mma_abT<D, 64>(tmem_base + kColdP + g * 128, smem_u32(sdO), vt);
-        mma_commit(s_full + g);
-      };
-      auto wait_kv = [&](int j) {
-        mbar_wait_spin(k_full + j % kDqKStages, (j / kDqKStages) & 1, abort_flag);
-        mbar_wait_spin(v_full + j % kDqVStages, (j / kDqVStages) & 1, abort_flag);
+      auto issue_s = [&](int j) {  // buffer j & 1 is free: both groups published dS(j-2) after loading S(j-2)
+        const int st = j % kDqKStages;
+        mbar_wait_spin(k_full + st, (j / kDqKStages) & 1, abort_flag);
         tc_fence_after_sync();
+        mma_abT<D>(tmem_base + kColS + (j & 1) * 128, smem_u32(sQ), smem_u32(sK + st * TileGeom<D>::kBytes));
+        mma_commit(s_full + (j & 1));
       };
-      auto issue_dq = [&](int j, int g) {
-        mbar_wait_spin(ds_full + g, j & 1, abort_flag);
+      auto issue_dp = [&](int j) {  // overwrites dS(j-1): issued after the dQ MMAs that read it, MMAs run in order
+        const int st = j % kDqVStages;
+        mbar_wait_spin(v_full + st, (j / kDqVStages) & 1, abort_flag);
         tc_fence_after_sync();
-        const uint32_t kt = smem_u32(sK + (j % kDqKStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
-        mma_pb<D, 64>(tmem_base + kColdQ, tmem_base + kColdS + g * 32, kt, j > 0 || g > 0);
+        mma_abT<D>(tmem_base + kColdP, smem_u32(sdO), smem_u32(sV + st * TileGeom<D>::kBytes));
+        mma_commit(v_empty + st);
+        mma_commit(dp_full);
       };
       mbar_wait_spin(q_full, 0, abort_flag);
-      wait_kv(0);
-      issue_sdp(0, 0);
-      issue_sdp(0, 1);
-      mma_commit(v_empty + 0);
+      issue_s(0);
+      issue_dp(0);
+      if (n_tiles > 1) issue_s(1);
       for (int j = 0; j < n_tiles; ++j) {
-        issue_dq(j, 0);
-        if (j + 1 < n_tiles) {
-          wait_kv(j + 1);
-          issue_sdp(j + 1, 0);
-        }
-        issue_dq(j, 1);
-        mma_commit(k_empty + j % kDqKStages);
-        if (j + 1 < n_tiles) {
-          issue_sdp(j + 1, 1);
-          mma_commit(v_empty + (j + 1) % kDqVStages);
-        }
+        const int st = j % kDqKStages;
+        const uint32_t kt = smem_u32(sK + st * TileGeom<D>::kBytes);
+        mbar_wait_spin(ds_full, j & 1, abort_flag);
+        tc_fence_after_sync();
+        mma_pb<D, 64>(tmem_base + kColdQ, tmem_base + kColdP, kt, j > 0);
+        mma_pb<D, 64>(tmem_base + kColdQ, tmem_base + kColdP + 64, kt + kHalfBytes, true);
+        mma_commit(k_empty + st);
+        if (j + 1 < n_tiles) issue_dp(j + 1);
+        if (j + 2 < n_tiles) issue_s(j + 2);
       }
       mma_commit(dq_full);
     }
@@ -195,39 +208,65 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const float lse2 = in_range ? lse[stat_idx] * kLog2e : 0.f;
     const float delta_r = in_range ? delta[stat_idx] : 0.f;
     const float scale_log2 = scale * kLog2e;
+    const uint64_t sc2 = f32x2(scale_log2, scale_log2), nl2 = f32x2(-lse2, -lse2), nd2 = f32x2(-delta_r, -delta_r);
     int j = 0;
     for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
-      const int valid = it.valid(segs) - 64 * g;  // valid keys of this group's half (may be <= 0)
-      mbar_wait(s_full + g, j & 1, abort_flag);
+      const int tile_valid = it.valid(segs);
+      const int valid = tile_valid - 64 * g;  // valid keys of this group's half (may be <= 0)
+      const uint32_t colS = kColS + (j & 1) * 128 + g * 64;
+      mbar_wait(s_full + (j & 1), (j >> 1) & 1, abort_flag);
       tc_fence_after_sync();
-      uint32_t s[2][32], dp[2][32], ds[32];
-      tmem_ld32(tmem_lane + kColS + g * 128, s[0]);
-      tmem_ld32(tmem_lane + kColS + g * 128 + 32, s[1]);
-      tmem_ld32(tmem_lane + kColdP + g * 128, dp[0]);
-      tmem_ld32(tmem_lane + kColdP + g * 128 + 32, dp[1]);
+      uint32_t s[2][32];
+      tmem_ld32(tmem_lane + colS, s[0]);
+      tmem_ld32(tmem_lane + colS + 32, s[1]);
       tmem_wait_ld();
+      // P = exp2(s * scale * log2e - LSE * log2e), kept as packed fp32 pairs in the registers of S
+      uint64_t p2[2][16];
 #pragma unroll
       for (int c2 = 0; c2 < 2; ++c2)
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(s[c2][c]), scale_log2, -lse2));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(s[c2][c + 1]), scale_log2, -lse2));
-          float d0 = p0 * (__uint_as_float(dp[c2][c]) - delta_r);
-          float d1 = p1 * (__uint_as_float(dp[c2][c + 1]) - delta_r);
-          if (valid < 64) {
+          const uint64_t x2 = fma2(f32x2(__uint_as_float(s[c2][c]), __uint_as_float(s[c2][c + 1])), sc2, nl2);
+          float p0, p1;
+          if (((c >> 1) & 7) < kDqPolyOf8) {
+            exp2_poly_pair(x2, p0, p1);
+          } else {
+            float x0, x1;
+            f32x2_split(x2, x0, x1);
+            p0 = fast_exp2(x0);
+            p1 = fast_exp2(x1);
+          }
+          p2[c2][c >> 1] = f32x2(p0, p1);
+        }
+      mbar_wait(dp_full, j & 1, abort_flag);
+      tc_fence_after_sync();
+#pragma unroll
+      for (int c2 = 0; c2 < 2; ++c2) {
+        uint32_t dp[32], ds[16];
+        tmem_ld32(tmem_lane + kColdP + g * 64 + c2 * 32, dp);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const uint64_t d2 = mul2(p2[c2][c >> 1],
+                                   add2(f32x2(__uint_as_float(dp[c]), __uint_as_float(dp[c + 1])), nd2));
+          float d0, d1;
+          f32x2_split(d2, d0, d1);
+          if (valid < 64) {  // stale keys past the segment's end: S and dP hold anything, dS must be 0
             if (c2 * 32 + c >= valid) d0 = 0.f;
             if (c2 * 32 + c + 1 >= valid) d1 = 0.f;
           }
-          ds[c2 * 16 + (c >> 1)] = pack_bf16(d0, d1);
+          ds[c >> 1] = pack_bf16(d0, d1);
         }
-      tmem_st32(tmem_lane + kColdS + g * 32, ds);
+        // in place: the 16 packed columns written here lie inside the 32 dP columns just read (c2 = 0) or
+        // inside columns read one step earlier (c2 = 1), all owned by this thread
+        tmem_st16(tmem_lane + kColdP + g * 64 + c2 * 16, ds);
+      }
       // Key rows past the segment's end may hold stale cache contents: dS is 0 there, but 0 * NaN is NaN.
-      // Group 0 clears them (all 128 rows' worth) before it publishes dS_0, which both dQ MMAs wait for.
-      if (g == 0 && it.valid(segs) < kTile)
-        zero_tile_rows_from<D>(sK + (j % kDqKStages) * TileGeom<D>::kBytes, it.valid(segs), r);
+      if (g == 0 && tile_valid < kTile)
+        zero_tile_rows_from<D>(sK + (j % kDqKStages) * TileGeom<D>::kBytes, tile_valid, r);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(ds_full + g);
+      mbar_arrive(ds_full);
     }
     // ---- epilogue: group g writes columns [g D/2, (g+1) D/2) of dQ
     mbar_wait(dq_full, 0, abort_flag);
