@@ -283,13 +283,16 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 // ------------------------------------------------------------------------------------------ dK, dV
 // Warp-specialised, one CTA (one 128-key tile of the chunk) per SM; K and V of the tile stay in shared
 // memory and the query tiles stream through a 2-deep ring of (Q, dO) pairs:
-//   warps 0-3  group 0: queries  0..63 of every query tile    warps 4-7  group 1: queries 64..127
+//   warps 0-3  group 0: queries  0..63 of every query tile (one key row per thread)
+//   warps 4-7  group 1: queries 64..127
 //   warp  8    MMA issuer                                       warp  9    TMA producer
-// Per query tile and group g: S^T_g = K Q_g^T and dP^T_g = V dO_g^T (128 keys x 64 queries; one key row per
-// thread), P^T_g and dS^T_g are written over them as bf16, then dV += P^T_g dO_g and dK += dS^T_g Q_g.
-//   TMEM columns: S^T0 [0,64) dP^T0 [64,128) S^T1 [128,192) dP^T1 [192,256) dK [256,256+D) dV [384,384+D)
+// Per query tile i: S^T = K Q^T and dP^T = V dO^T are full 128x128 MMAs (keys x queries).  A thread turns its
+// 64 S^T values into P^T (bf16 pairs written over its own S^T columns) -> dV += P^T dO and S^T(i+1) follow;
+// then dP^T into dS^T = P^T o (dP^T - delta) in place -> dK += dS^T Q and dP^T(i+1) follow.
+//   TMEM columns: S^T / P^T [0,128)  dP^T / dS^T [128,256)  dK [256,256+D)  dV [384,384+D)
 constexpr int kDkvStages = 2;
 constexpr int kDkvThreads = 320;
+constexpr int kDkvPolyOf8 = 2;
 
 template <int D> struct DkvSmem {
   static constexpr int kK = 0;
@@ -319,16 +322,18 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
   uint64_t* kv_full = bars;
   uint64_t* q_full = bars + 1;                 // [kDkvStages]
   uint64_t* q_empty = q_full + kDkvStages;
-  uint64_t* s_full = q_empty + kDkvStages;     // [2]
-  uint64_t* p_full = s_full + 2;               // [2]
-  uint64_t* acc_full = p_full + 2;
+  uint64_t* s_full = q_empty + kDkvStages;
+  uint64_t* dp_full = s_full + 1;
+  uint64_t* p_full = dp_full + 1;              // 256 arrivals
+  uint64_t* ds_full = p_full + 1;              // 256 arrivals
+  uint64_t* acc_full = ds_full + 1;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int k0 = blockIdx.x * kTile, h = blockIdx.y, b = blockIdx.z;
   constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kColSt = 0, kColdPt = 64 /* + 128 g */, kColdK = 256, kColdV = 384;
+  constexpr uint32_t kColSt = 0, kColdPt = 128, kColdK = 256, kColdV = 384;
   constexpr int kMmaWarp = 8, kTmaWarp = 9;
   constexpr int kHalfBytes = 64 * 128;
   const int n_tiles = (n_q + kTile - 1) / kTile;
@@ -336,7 +341,10 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
   if (tid == 0) {
     mbar_init(kv_full, 1);
     for (int i = 0; i < kDkvStages; ++i) { mbar_init(q_full + i, 1); mbar_init(q_empty + i, 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 128); }
+    mbar_init(s_full, 1);
+    mbar_init(dp_full, 1);
+    mbar_init(p_full, 256);
+    mbar_init(ds_full, 256);
     mbar_init(acc_full, 1);
     *abort_flag = 0;
     fence_mbar_init();
@@ -366,38 +374,37 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     }
   } else if (warp == kMmaWarp) {
     if (lane == 0) {
-      auto issue_sdp = [&](int i, int g) {
-        const uint32_t qt = smem_u32(sQ + (i % kDkvStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
-        const uint32_t dot = smem_u32(sdO + (i % kDkvStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
-        mma_abT<D, 64>(tmem_base + kColSt + g * 128, smem_u32(sK), qt);
-        mma_abT<D, 64>(tmem_base + kColdPt + g * 128, smem_u32(sV), dot);
-        mma_commit(s_full + g);
-      };
-      auto issue_acc = [&](int i, int g) {
-        mbar_wait_spin(p_full + g, i & 1, abort_flag);
-        tc_fence_after_sync();
-        const uint32_t qt = smem_u32(sQ + (i % kDkvStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
-        const uint32_t dot = smem_u32(sdO + (i % kDkvStages) * TileGeom<D>::kBytes) + g * kHalfBytes;
-        mma_pb<D, 64>(tmem_base + kColdV, tmem_base + kColSt + g * 128, dot, i > 0 || g > 0);
-        mma_pb<D, 64>(tmem_base + kColdK, tmem_base + kColdPt + g * 128, qt, i > 0 || g > 0);
-      };
+      auto q_tile = [&](int i) { return smem_u32(sQ + (i % kDkvStages) * TileGeom<D>::kBytes); };
+      auto do_tile = [&](int i) { return smem_u32(sdO + (i % kDkvStages) * TileGeom<D>::kBytes); };
       auto wait_q = [&](int i) {
         mbar_wait_spin(q_full + i % kDkvStages, (i / kDkvStages) & 1, abort_flag);
         tc_fence_after_sync();
       };
       mbar_wait_spin(kv_full, 0, abort_flag);
       wait_q(0);
-      issue_sdp(0, 0);
-      issue_sdp(0, 1);
+      mma_abT<D>(tmem_base + kColSt, smem_u32(sK), q_tile(0));
+      mma_commit(s_full);
+      mma_abT<D>(tmem_base + kColdPt, smem_u32(sV), do_tile(0));
+      mma_commit(dp_full);
       for (int i = 0; i < n_tiles; ++i) {
-        issue_acc(i, 0);
-        if (i + 1 < n_tiles) {
+        mbar_wait_spin(p_full, i & 1, abort_flag);
+        tc_fence_after_sync();
+        mma_pb<D, 64>(tmem_base + kColdV, tmem_base + kColSt, do_tile(i), i > 0);
+        mma_pb<D, 64>(tmem_base + kColdV, tmem_base + kColSt + 64, do_tile(i) + kHalfBytes, true);
+        if (i + 1 < n_tiles) {  // overwrites P^T(i) after the dV MMAs that read it (MMAs run in order)
           wait_q(i + 1);
-          issue_sdp(i + 1, 0);
+          mma_abT<D>(tmem_base + kColSt, smem_u32(sK), q_tile(i + 1));
+          mma_commit(s_full);
         }
-        issue_acc(i, 1);
+        mbar_wait_spin(ds_full, i & 1, abort_flag);
+        tc_fence_after_sync();
+        mma_pb<D, 64>(tmem_base + kColdK, tmem_base + kColdPt, q_tile(i), i > 0);
+        mma_pb<D, 64>(tmem_base + kColdK, tmem_base + kColdPt + 64, q_tile(i) + kHalfBytes, true);
         mma_commit(q_empty + i % kDkvStages);
-        if (i + 1 < n_tiles) issue_sdp(i + 1, 1);
+        if (i + 1 < n_tiles) {
+          mma_abT<D>(tmem_base + kColdPt, smem_u32(sV), do_tile(i + 1));
+          mma_commit(dp_full);
+        }
       }
       mma_commit(acc_full);
     }
@@ -406,6 +413,7 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const int r = tid & 127;  // key row inside the tile = TMEM lane
     const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const float scale_log2 = scale * kLog2e;
+    const uint64_t sc2 = f32x2(scale_log2, scale_log2);
     const size_t stat_base = (static_cast<size_t>(b) * heads + h) * n_q;
     for (int i = 0; i < n_tiles; ++i) {
       // per-query constants of this group's 64 queries; +inf as LSE turns rows past n_q into P = 0
@@ -416,32 +424,59 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
                            : make_float2(INFINITY, 0.f);
       }
       named_barrier_sync(1 + g, 128);
-      mbar_wait(s_full + g, i & 1, abort_flag);
+      mbar_wait(s_full, i & 1, abort_flag);
       tc_fence_after_sync();
-      uint32_t s[2][32], dp[2][32], pt[32], ds[32];
-      tmem_ld32(tmem_lane + kColSt + g * 128, s[0]);
-      tmem_ld32(tmem_lane + kColSt + g * 128 + 32, s[1]);
-      tmem_ld32(tmem_lane + kColdPt + g * 128, dp[0]);
-      tmem_ld32(tmem_lane + kColdPt + g * 128 + 32, dp[1]);
+      uint32_t s[2][32], pt[32];
+      tmem_ld32(tmem_lane + kColSt + g * 64, s[0]);
+      tmem_ld32(tmem_lane + kColSt + g * 64 + 32, s[1]);
       tmem_wait_ld();
+      uint64_t p2[2][16];
 #pragma unroll
       for (int c2 = 0; c2 < 2; ++c2)
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
           const float4 st2 = *reinterpret_cast<const float4*>(stat + c2 * 32 + c);  // (lse2, delta) x 2 queries
-          const float p0 = fast_exp2(fmaf(__uint_as_float(s[c2][c]), scale_log2, -st2.x));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(s[c2][c + 1]), scale_log2, -st2.z));
-          const float d0 = p0 * (__uint_as_float(dp[c2][c]) - st2.y);
-          const float d1 = p1 * (__uint_as_float(dp[c2][c + 1]) - st2.w);
+          const uint64_t x2 = fma2(f32x2(__uint_as_float(s[c2][c]), __uint_as_float(s[c2][c + 1])), sc2,
+                                   f32x2(-st2.x, -st2.z));
+          float p0, p1;
+          if (((c >> 1) & 7) < kDkvPolyOf8) {
+            exp2_poly_pair(x2, p0, p1);
+          } else {
+            float x0, x1;
+            f32x2_split(x2, x0, x1);
+            p0 = fast_exp2(x0);
+            p1 = fast_exp2(x1);
+          }
+          p2[c2][c >> 1] = f32x2(p0, p1);
           pt[c2 * 16 + (c >> 1)] = pack_bf16(p0, p1);
-          ds[c2 * 16 + (c >> 1)] = pack_bf16(d0, d1);
         }
-      // in place: every column of S^T_g and dP^T_g this thread owns is already in registers
-      tmem_st32(tmem_lane + kColSt + g * 128, pt);
-      tmem_st32(tmem_lane + kColdPt + g * 128, ds);
+      // in place: every S^T column this thread owns is already in registers
+      tmem_st32(tmem_lane + kColSt + g * 64, pt);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(p_full + g);
+      mbar_arrive(p_full);
+
+      mbar_wait(dp_full, i & 1, abort_flag);
+      tc_fence_after_sync();
+#pragma unroll
+      for (int c2 = 0; c2 < 2; ++c2) {
+        uint32_t dp[32], ds[16];
+        tmem_ld32(tmem_lane + kColdPt + g * 64 + c2 * 32, dp);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const float4 st2 = *reinterpret_cast<const float4*>(stat + c2 * 32 + c);
+          const uint64_t d2 = mul2(p2[c2][c >> 1], add2(f32x2(__uint_as_float(dp[c]), __uint_as_float(dp[c + 1])),
+                                                        f32x2(-st2.y, -st2.w)));
+          float d0, d1;
+          f32x2_split(d2, d0, d1);
+          ds[c >> 1] = pack_bf16(d0, d1);
+        }
+        tmem_st16(tmem_lane + kColdPt + g * 64 + c2 * 16, ds);
+      }
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(ds_full);
     }
     mbar_wait(acc_full, 0, abort_flag);
     tc_fence_after_sync();
