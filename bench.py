@@ -359,6 +359,139 @@ def run_ours(args):
     return 0
 
 
+# ----------------------------------------------------------------------------------------------- other workloads
+def _event_ms(fn, reps=1):
+    import torch
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    s.record()
+    for _ in range(reps):
+        fn()
+    e.record()
+    torch.cuda.synchronize()
+    return s.elapsed_time(e) / reps
+
+
+def run_extra(args):
+    """Rollout, clip-window update and context sweep on one GPU (device-resident inputs, CUDA events)."""
+    import torch
+    from paper_2603_17051_b200 import binding as A
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = measured_peaks()
+
+    def rnd(i, shape):
+        bits = synth.normal_bf16(synth.tensor_seed(9, i), shape)
+        return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    H, D, T, c = 12, 128, 1560, 3
+    M = c * T
+    if args.workload == "rollout":
+        w = synth.ROLLOUT
+        B, chunks, steps = w.batch, 80, 4
+        slots = w.window_frames if args.reading == "A" else w.window_frames + c
+        cache = A.astro_kvcache_create(B, H, D, T, w.sink_frames, slots, device=dev)
+        q, kc, vc = (rnd(i, (B, M, H, D)) for i in range(3))
+        o = torch.empty_like(q); lse = torch.empty((B, H, M), dtype=torch.float32, device=dev)
+        cap = w.sink_frames + slots
+
+        def rollout():
+            A.astro_kvcache_reset(cache)
+            flops = 0.0
+            for n in range(chunks):
+                sink, win, _ = A.astro_kvcache_query(cache)
+                over = sink + win - (cap - c)
+                if over > 0:
+                    A.astro_kvcache_evict(cache, over)
+                held = min(sink + win, cap - c)
+                for _ in range(steps):                       # denoising steps against a fixed cache
+                    A.astro_chunk_attn_fwd(cache, q, kc, vc, w.scale, o=o, lse=lse)
+                flops += steps * 4.0 * B * H * M * (held * T + M) * D
+                A.astro_kvcache_append(cache, kc, vc, c)     # one clean-frame K/V write
+            return flops
+        rollout()
+        torch.cuda.synchronize()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record(); flops = rollout(); e.record(); torch.cuda.synchronize()
+        ms = s.elapsed_time(e)
+        A.astro_last_device_status()
+        frames = chunks * c
+        print(json.dumps({"workload": "rollout", "reading": args.reading, "metric": "rollout_latent_frames_per_s",
+                          "value": frames * B / (ms * 1e-3), "unit": "latent-frames/s (all %d samples)" % B,
+                          "per_sample_latent_frames_per_s": frames / (ms * 1e-3), "ms_total": ms,
+                          "tflops": flops / (ms * 1e-3) / 1e12, "keys_steady_state": (cap - c) * T + M,
+                          "config": "B=4 H=12 D=128 T=1560, S=3 + %d window slots, 80 chunks x (evict, 4 fwd, append)" % slots,
+                          "frac_of_bf16_sustained": flops / (ms * 1e-3) / 1e12 / peaks["bf16_sustained"]}))
+        return 0
+    if args.workload == "rl_update":
+        w = synth.RL_UPDATE
+        B = w.batch
+        cache = A.astro_kvcache_create(B, H, D, T, w.sink_frames, w.window_frames, device=dev)
+        A.astro_kvcache_append(cache, rnd(10, (B, w.ctx_tokens, H, D)), rnd(11, (B, w.ctx_tokens, H, D)), w.held_frames)
+        q, kc, vc, do = (rnd(i, (B, M, H, D)) for i in range(4))
+        o = torch.empty_like(q); lse = torch.empty((B, H, M), dtype=torch.float32, device=dev)
+        dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+        ws = torch.empty(A.astro_chunk_attn_bwd_workspace_bytes(B, H, M, D), dtype=torch.uint8, device=dev)
+        fwd = lambda: A.astro_chunk_attn_fwd(cache, q, kc, vc, w.scale, o=o, lse=lse)
+        bwd = lambda: A.astro_chunk_attn_bwd(cache, q, kc, vc, o, lse, do, w.scale, dq=dq, dk_chunk=dk, dv_chunk=dv,
+                                             workspace=ws)
+        for _ in range(5):
+            fwd(); bwd()
+        ms_f, ms_b = _event_ms(fwd, 20), _event_ms(bwd, 20)
+        A.astro_last_device_status()
+        tf = lambda fl, ms: fl / (ms * 1e-3) / 1e12
+        print(json.dumps({"workload": "rl_update", "metric": "chunk_attn_fwd_bwd_tflops", "unit": "TFLOP/s",
+                          "value": tf(w.fwd_flops() + w.bwd_flops(), ms_f + ms_b),
+                          "fwd": {"ms": ms_f, "tflops": tf(w.fwd_flops(), ms_f)},
+                          "bwd": {"ms": ms_b, "tflops": tf(w.bwd_flops(), ms_b)},
+                          "config": "B=2 H=12 D=128, 4680 q/k with grads over 28080 detached keys",
+                          "frac_of_bf16_sustained": tf(w.fwd_flops() + w.bwd_flops(), ms_f + ms_b) / peaks["bf16_sustained"],
+                          "frac_of_bf16_burst": tf(w.fwd_flops() + w.bwd_flops(), ms_f + ms_b) / peaks["bf16_burst"]}))
+        return 0
+    # sweep: 30 independent layers x 8 samples x 7 chunks x 4 denoising steps, keys per query held fixed
+    B, layers, chunks, steps = 8, 30, 7, 4
+    q, kc, vc = (rnd(i, (B, M, H, D)) for i in range(3))
+    o = torch.empty_like(q); lse = torch.empty((B, H, M), dtype=torch.float32, device=dev)
+    scale = 1.0 / float(np.sqrt(D))
+    for n_k in synth.SWEEP_KEYS:
+        n_ctx = max(n_k - M, 0)
+        n_kc = min(n_k, M)
+        caches = []
+        if n_ctx:
+            tpf = 780                                          # half frames, so 16380 keys (10.5 frames) fit exactly
+            frames = n_ctx // tpf
+            per_cache = 2 * B * H * n_ctx * D * 2
+            n_alloc = layers if per_cache * layers < 120e9 else 1
+            fill_k, fill_v = rnd(20, (B, n_ctx, H, D)), rnd(21, (B, n_ctx, H, D))
+            for _ in range(n_alloc):
+                cch = A.astro_kvcache_create(B, H, D, tpf, 0, frames, device=dev)
+                A.astro_kvcache_append(cch, fill_k, fill_v, frames)
+                caches.append(cch)
+            del fill_k, fill_v
+        kcs, vcs = kc[:, :n_kc].contiguous(), vc[:, :n_kc].contiguous()
+
+        def sweep_pass():
+            for _ in range(chunks):
+                for _ in range(steps):
+                    for layer in range(layers):
+                        cch = caches[layer % len(caches)] if caches else None
+                        A.astro_chunk_attn_fwd(cch, q, kcs, vcs, scale, o=o, lse=lse)
+        for layer in range(min(layers, 3)):
+            A.astro_chunk_attn_fwd(caches[layer % len(caches)] if caches else None, q, kcs, vcs, scale, o=o, lse=lse)
+        ms = _event_ms(sweep_pass, 1)
+        A.astro_last_device_status()
+        flops = 4.0 * B * H * M * (n_ctx + n_kc) * D * layers * chunks * steps
+        print(json.dumps({"workload": "sweep", "keys": n_k, "metric": "rollout_latent_frames_per_s",
+                          "value": chunks * c * B / (ms * 1e-3), "unit": "latent-frames/s (all 8 samples)",
+                          "per_sample_latent_frames_per_s": chunks * c / (ms * 1e-3), "ms_total": ms,
+                          "tflops": flops / (ms * 1e-3) / 1e12,
+                          "frac_of_bf16_sustained": flops / (ms * 1e-3) / 1e12 / peaks["bf16_sustained"],
+                          "caches_resident": len(caches), "note": "attention only; 30 layers x 7 chunks x 4 steps"}))
+        del caches
+        torch.cuda.empty_cache()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -366,8 +499,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", choices=("layer", "rollout", "rl_update", "sweep"), default="layer",
+                    help="layer (default): the contract line; the others print one JSON line per extra workload")
+    ap.add_argument("--reading", choices=("A", "B"), default="A",
+                    help="rollout only: A = window capacity counts the chunk (12 held + chunk), B = 15 held + chunk")
     args = ap.parse_args()
-    return run_reference(args) if args.impl == "reference" else run_ours(args)
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.workload != "layer":
+        return run_extra(args)
+    return run_ours(args)
 
 
 if __name__ == "__main__":
