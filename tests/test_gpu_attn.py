@@ -235,3 +235,60 @@ def test_rl_update_shape_backward_sampled():
                     (dq_ref, dk_ref, dv_ref), tag="b%d h%d" % (b, h))
         e = rel_l2(f64(dq[b:b + 1, rows, h:h + 1]), dq_ref[:, rows])
         assert e <= 1e-2, "sampled dQ rows rel-L2 %.3e" % e
+
+
+def test_rollout_shape_streamed_eight_chunks_sampled():
+    """Long-rollout shape (batch 4, per-sample caches, 3 sink + 12 window slots, 1560 tokens per frame):
+    eight chunks streamed so that the ring wraps; cache bit-exact, forward of the last chunk on sampled rows."""
+    from paper_2603_17051_b200 import binding as A
+    w = synth.ROLLOUT
+    H, D, T, c, M = w.heads, w.head_dim, w.tokens_per_frame, w.chunk_frames, w.chunk_tokens
+    cache = A.astro_kvcache_create(w.batch, H, D, T, w.sink_frames, w.window_frames)
+    model = orc.RollingKVCache(w.sink_frames, w.window_frames)
+    cap = w.sink_frames + w.window_frames
+    for n in range(8):
+        over = model.held() - (cap - c)
+        if over > 0:
+            A.astro_kvcache_evict(cache, over); model.evict(over)
+        kb = synth.normal_bf16(synth.tensor_seed(3, 2 * n), (w.batch, M, H, D))
+        vb = synth.normal_bf16(synth.tensor_seed(3, 2 * n + 1), (w.batch, M, H, D))
+        kc, vc = dev_bf16(kb), dev_bf16(vb)
+        if n == 7:
+            qb = synth.normal_bf16(synth.tensor_seed(3, 100), (w.batch, M, H, D))
+            q = dev_bf16(qb)
+            for _ in range(4):                                   # four denoising steps against a fixed cache
+                o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, w.scale)
+            A.astro_last_device_status()
+            assert model.held() == 12
+            mk, mv = model.export()
+            rows = _sample_rows(M, 48, np.random.default_rng(3))
+            for (b, h) in ((0, 0), (3, 7)):
+                sl = lambda x: orc.bf16_bits_to_f64(x[b:b + 1, :, h:h + 1, :])
+                o_ref, lse_ref = orc.chunk_attn_fwd(sl(qb)[:, rows], sl(mk), sl(mv), sl(kb), sl(vb), w.scale)
+                check_fwd(o[b:b + 1, rows, h:h + 1], lse[b:b + 1, h:h + 1][:, :, rows], o_ref, lse_ref, tag="b%d h%d" % (b, h))
+        A.astro_kvcache_append(cache, kc, vc, c); model.append(kb, vb, T)
+    ke, ve = A.astro_kvcache_export(cache)
+    mk, mv = model.export()
+    assert np.array_equal(host_bits(ke), mk) and np.array_equal(host_bits(ve), mv)
+    assert A.astro_kvcache_query(cache) == (3, 12, 24)
+
+
+def test_longest_sweep_context_sampled():
+    """65520 keys per query (60840 cached as 78 half-frames of 780 tokens + the 4680-token chunk), batch 2 of the
+    sweep's 8 samples: forward on sampled rows."""
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, T, frames, M = 2, 12, 128, 780, 78, 4680
+    cache = A.astro_kvcache_create(B, H, D, T, 0, frames)
+    kxb = synth.normal_bf16(synth.tensor_seed(5, 0), (B, frames * T, H, D))
+    vxb = synth.normal_bf16(synth.tensor_seed(5, 1), (B, frames * T, H, D))
+    A.astro_kvcache_append(cache, dev_bf16(kxb), dev_bf16(vxb), frames)
+    bits = [synth.normal_bf16(synth.tensor_seed(5, 10 + i), (B, M, H, D)) for i in range(3)]
+    q, kc, vc = (dev_bf16(x) for x in bits)
+    scale = 1.0 / np.sqrt(D)
+    o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, scale)
+    A.astro_last_device_status()
+    rows = _sample_rows(M, 48, np.random.default_rng(5))
+    for (b, h) in ((0, 5), (1, 11)):
+        sl = lambda x: orc.bf16_bits_to_f64(x[b:b + 1, :, h:h + 1, :])
+        o_ref, lse_ref = orc.chunk_attn_fwd(sl(bits[0])[:, rows], sl(kxb), sl(vxb), sl(bits[1]), sl(bits[2]), scale)
+        check_fwd(o[b:b + 1, rows, h:h + 1], lse[b:b + 1, h:h + 1][:, :, rows], o_ref, lse_ref, tag="b%d h%d" % (b, h))
