@@ -416,7 +416,17 @@ def run_extra(args):
         ms = s.elapsed_time(e)
         A.astro_last_device_status()
         frames = chunks * c
-        print(json.dumps({"workload": "rollout", "reading": args.reading, "metric": "rollout_latent_frames_per_s",
+        # append alone: 3 frames of K and V for all samples, read + written once (L2 flushed before each)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        t_app = []
+        for _ in range(20):
+            A.astro_kvcache_reset(cache); flush.zero_()
+            t_app.append(_event_ms(lambda: A.astro_kvcache_append(cache, kc, vc, c)))
+        app_ms = float(np.median(t_app[3:]))
+        app_bytes = 2 * 2 * B * H * c * T * D * 2
+        print(json.dumps({"workload": "rollout", "reading": args.reading,
+                          "append": {"ms": app_ms, "bytes_moved": app_bytes, "gbs": app_bytes / app_ms / 1e6,
+                                     "frac_of_hbm": app_bytes / app_ms / 1e6 / peaks["hbm"]}, "metric": "rollout_latent_frames_per_s",
                           "value": frames * B / (ms * 1e-3), "unit": "latent-frames/s (all %d samples)" % B,
                           "per_sample_latent_frames_per_s": frames / (ms * 1e-3), "ms_total": ms,
                           "tflops": flops / (ms * 1e-3) / 1e12, "keys_steady_state": (cap - c) * T + M,

@@ -229,19 +229,20 @@ astro_status_t launch_ring_copy(const astro_kvcache* c, void* k_user, void* v_us
                                 cudaStream_t st) {
   const auto& d = c->d;
   const int vpr = d.head_dim * 2 / 16;
-  const long long per_frame = static_cast<long long>(d.tokens_per_frame) * d.heads * vpr;
-  if (per_frame * kMaxFramesPerCopy >= (1ll << 31)) return ASTRO_ERR_SHAPE;
+  const int row_vecs = d.heads * vpr;
+  const int threads = row_vecs >= 256 ? 256 : ((row_vecs + 31) / 32) * 32;
+  const int chunks_per_frame = (d.tokens_per_frame + kRingTokensPerThread - 1) / kRingTokensPerThread;
+  if (d.cache_batch > 32767 || static_cast<long long>(chunks_per_frame) * kMaxFramesPerCopy > 65535)
+    return ASTRO_ERR_SHAPE;
   for (int f0 = 0; f0 < n_frames; f0 += kMaxFramesPerCopy) {
     SlotMap map;
     map.n = n_frames - f0 < kMaxFramesPerCopy ? n_frames - f0 : kMaxFramesPerCopy;
     for (int j = 0; j < map.n; ++j) map.slot[j] = slots[f0 + j];
-    const long long vec_per_batch = per_frame * map.n;
-    const long long total = vec_per_batch * d.cache_batch;
-    dim3 grid(static_cast<unsigned>((total + 1023) / 1024), 2, 1);
-    ring_copy_kernel<ToCache><<<grid, 256, 0, st>>>(
+    dim3 grid((row_vecs + threads - 1) / threads, map.n * chunks_per_frame, 2 * d.cache_batch);
+    ring_copy_kernel<ToCache><<<grid, threads, 0, st>>>(
         static_cast<uint4*>(k_user), static_cast<uint4*>(v_user), static_cast<uint4*>(c->k),
         static_cast<uint4*>(c->v), map, d.heads, d.tokens_per_frame, vpr, d.sink_frames + d.window_frames, f0,
-        n_frames, vec_per_batch, total);
+        n_frames, chunks_per_frame);
   }
   return launch_status();
 }
