@@ -433,6 +433,31 @@ def run_extra(args):
                           "config": "B=4 H=12 D=128 T=1560, S=3 + %d window slots, 80 chunks x (evict, 4 fwd, append)" % slots,
                           "frac_of_bf16_sustained": flops / (ms * 1e-3) / 1e12 / peaks["bf16_sustained"]}))
         return 0
+    if args.workload == "group":
+        # clip-level group-wise sampling: G candidate chunks decode against one frozen, shared prefix
+        w = synth.LAYER_FWD
+        G = args.group
+        Bc = G if args.replicated else 1
+        cache = A.astro_kvcache_create(Bc, H, D, T, w.sink_frames, w.window_frames, device=dev)
+        kx, vx = rnd(10, (1, w.ctx_tokens, H, D)), rnd(11, (1, w.ctx_tokens, H, D))
+        if args.replicated:
+            kx, vx = kx.expand(G, -1, -1, -1).contiguous(), vx.expand(G, -1, -1, -1).contiguous()
+        A.astro_kvcache_append(cache, kx, vx, w.held_frames)
+        del kx, vx
+        q, kc, vc = (rnd(i, (G, M, H, D)) for i in range(3))
+        o = torch.empty_like(q); lse = torch.empty((G, H, M), dtype=torch.float32, device=dev)
+        fwd = lambda: A.astro_chunk_attn_fwd(cache, q, kc, vc, w.scale, o=o, lse=lse)
+        for _ in range(3):
+            fwd()
+        ms = _event_ms(fwd, args.steps if args.steps < 50 else 10)
+        A.astro_last_device_status()
+        flops = G * w.fwd_flops()
+        print(json.dumps({"workload": "group", "G": G, "prefix": "replicated" if args.replicated else "shared",
+                          "metric": "chunk_attn_fwd_tflops", "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                          "ms": ms, "cache_bytes": 2 * Bc * H * (w.sink_frames + w.window_frames) * T * D * 2,
+                          "config": "G x (4680 q, 12 heads, D=128) over 28080 cached + 4680 chunk keys",
+                          "frac_of_bf16_sustained": flops / (ms * 1e-3) / 1e12 / peaks["bf16_sustained"]}))
+        return 0
     if args.workload == "rl_update":
         w = synth.RL_UPDATE
         B = w.batch
@@ -509,8 +534,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", choices=("layer", "rollout", "rl_update", "sweep"), default="layer",
+    ap.add_argument("--workload", choices=("layer", "rollout", "rl_update", "sweep", "group"), default="layer",
                     help="layer (default): the contract line; the others print one JSON line per extra workload")
+    ap.add_argument("--group", type=int, default=24, help="group workload: candidates G decoding against one prefix")
+    ap.add_argument("--replicated", action="store_true",
+                    help="group workload: give every candidate its own copy of the prefix (comparison)")
     ap.add_argument("--reading", choices=("A", "B"), default="A",
                     help="rollout only: A = window capacity counts the chunk (12 held + chunk), B = 15 held + chunk")
     args = ap.parse_args()

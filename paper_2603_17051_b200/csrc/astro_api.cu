@@ -176,9 +176,10 @@ astro_status_t launch_fwd(const AttnArgs& a, const CUtensorMap& tq, const CUtens
   static bool done[64];
   astro_status_t s = set_smem_once(chunk_attn_fwd_kernel<D>, FwdSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
-  dim3 grid((a.n_q + kTile - 1) / kTile, a.heads, a.batch);
+  const int shared = (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
+  dim3 grid((a.n_q + kTile - 1) / kTile, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
   chunk_attn_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kTotal, st>>>(
-      tq, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0,
+      tq, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared,
       scale * kLog2e, static_cast<__nv_bfloat16*>(o), lse);
   return launch_status();
 }
@@ -201,10 +202,10 @@ astro_status_t launch_bwd_dq(const AttnArgs& a, const CUtensorMap& tq, const CUt
   static bool done[64];
   astro_status_t s = set_smem_once(chunk_attn_bwd_dq_kernel<D>, DqSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
-  dim3 grid_q((a.n_q + kTile - 1) / kTile, a.heads, a.batch);
+  const int shared = (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
+  dim3 grid_q((a.n_q + kTile - 1) / kTile, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
   chunk_attn_bwd_dq_kernel<D><<<grid_q, kDqThreads, DqSmem<D>::kTotal, st>>>(
-      tq, tdo, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads,
-      (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0, scale, lse, delta,
+      tq, tdo, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared, scale, lse, delta,
       static_cast<__nv_bfloat16*>(dq));
   return launch_status();
 }

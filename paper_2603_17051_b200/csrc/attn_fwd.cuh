@@ -58,7 +58,10 @@ chunk_attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int q0 = blockIdx.x * kTile, h = blockIdx.y, b = blockIdx.z;
+  // With one shared cache (frozen prefix of a sample group) the samples of a head are launched next to each
+  // other, so the head's cached K/V is fetched from HBM once and served to the whole group out of L2.
+  const int q0 = blockIdx.x * kTile;
+  const int h = cache_shared ? blockIdx.z : blockIdx.y, b = cache_shared ? blockIdx.y : blockIdx.z;
   const int bx = cache_shared ? 0 : b;
   constexpr uint32_t kTmemCols = 512;
   constexpr uint32_t kColS = 0 /* + 128 * buffer */, kColO = 256 /* + 128 * group */;
