@@ -90,6 +90,20 @@ astro_status_t astro_kvcache_evict(astro_kvcache_t* cache, int n_frames, void* s
 astro_status_t astro_kvcache_query(const astro_kvcache_t* cache, int* sink_held, int* window_held,
                                    int64_t* frames_seen);
 
+/* Checkpoint / resume.  The cache's whole state is the caller's storage plus this small record: a caller
+ * that saves both (Sec. 3.3: the forward roll that accumulates the cache is the expensive part of a
+ * training step) can later bind the saved bytes to a new handle with astro_kvcache_create and restore the
+ * record with astro_kvcache_set_state.  HOST pointers.  set_state returns ASTRO_ERR_SHAPE if the record
+ * does not fit the descriptor (counts out of range, window frames without a full sink). */
+typedef struct {
+  int sink_held;       /* frames in the sink slots */
+  int window_head;     /* ring index of the oldest window frame, 0..L-1 */
+  int window_held;     /* frames in the window ring */
+  int64_t frames_seen; /* frames appended since create/reset */
+} astro_kvcache_state_t;
+astro_status_t astro_kvcache_get_state(const astro_kvcache_t* cache, astro_kvcache_state_t* state);
+astro_status_t astro_kvcache_set_state(astro_kvcache_t* cache, const astro_kvcache_state_t* state);
+
 /* Inspection aid: write the held frames in logical order (sink frames, then
  * window oldest to newest) to k_out, v_out: device bf16 [B_c, held*T, H, D]. */
 astro_status_t astro_kvcache_export(const astro_kvcache_t* cache, void* k_out, void* v_out, void* stream);

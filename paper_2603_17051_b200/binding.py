@@ -16,7 +16,7 @@ STATUS_NAMES = {0: "ASTRO_OK", 1: "ASTRO_ERR_NULL", 2: "ASTRO_ERR_SHAPE", 3: "AS
                 4: "ASTRO_ERR_CAPACITY", 5: "ASTRO_ERR_UNDERFLOW", 6: "ASTRO_ERR_ARCH", 7: "ASTRO_ERR_CUDA",
                 8: "ASTRO_ERR_TIMEOUT"}
 
-EXPORTED = ("astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcache_destroy", "astro_kvcache_reset",
+EXPORTED = ("astro_kvcache_get_state", "astro_kvcache_set_state", "astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcache_destroy", "astro_kvcache_reset",
             "astro_kvcache_append", "astro_kvcache_evict", "astro_kvcache_query", "astro_kvcache_export",
             "astro_chunk_attn_fwd", "astro_chunk_attn_bwd_workspace_bytes", "astro_chunk_attn_bwd",
             "astro_chunk_attn_bwd_delta", "astro_chunk_attn_bwd_dq", "astro_chunk_attn_bwd_dkv",
@@ -34,6 +34,11 @@ class AstroError(RuntimeError):
 class KVCacheDesc(C.Structure):
     _fields_ = [("cache_batch", C.c_int), ("heads", C.c_int), ("head_dim", C.c_int),
                 ("tokens_per_frame", C.c_int), ("sink_frames", C.c_int), ("window_frames", C.c_int)]
+
+
+class KVCacheState(C.Structure):
+    _fields_ = [("sink_held", C.c_int), ("window_head", C.c_int), ("window_held", C.c_int),
+                ("frames_seen", C.c_int64)]
 
 
 _lib = None
@@ -61,6 +66,10 @@ def lib():
     L.astro_kvcache_evict.argtypes = [vp, ci, vp]
     L.astro_kvcache_query.restype = ci
     L.astro_kvcache_query.argtypes = [vp, C.POINTER(ci), C.POINTER(ci), C.POINTER(C.c_int64)]
+    L.astro_kvcache_get_state.restype = ci
+    L.astro_kvcache_get_state.argtypes = [vp, C.POINTER(KVCacheState)]
+    L.astro_kvcache_set_state.restype = ci
+    L.astro_kvcache_set_state.argtypes = [vp, C.POINTER(KVCacheState)]
     L.astro_kvcache_export.restype = ci
     L.astro_kvcache_export.argtypes = [vp, vp, vp, vp]
     L.astro_chunk_attn_fwd.restype = ci
@@ -175,6 +184,16 @@ def astro_kvcache_query(cache: KVCache):
     a, b, c = C.c_int(), C.c_int(), C.c_int64()
     _check(lib().astro_kvcache_query(cache.handle, C.byref(a), C.byref(b), C.byref(c)), "astro_kvcache_query")
     return a.value, b.value, c.value
+
+
+def astro_kvcache_get_state(cache: KVCache) -> KVCacheState:
+    st = KVCacheState()
+    _check(lib().astro_kvcache_get_state(cache.handle, C.byref(st)), "astro_kvcache_get_state")
+    return st
+
+
+def astro_kvcache_set_state(cache: KVCache, state: KVCacheState) -> None:
+    _check(lib().astro_kvcache_set_state(cache.handle, C.byref(state)), "astro_kvcache_set_state")
 
 
 def astro_kvcache_export(cache: KVCache, stream=None):

@@ -336,6 +336,29 @@ astro_status_t astro_kvcache_query(const astro_kvcache_t* c, int* sink_held, int
   return ASTRO_OK;
 }
 
+astro_status_t astro_kvcache_get_state(const astro_kvcache_t* c, astro_kvcache_state_t* state) {
+  if (!c || !state) return ASTRO_ERR_NULL;
+  state->sink_held = c->sink_held;
+  state->window_head = c->win_head;
+  state->window_held = c->win_held;
+  state->frames_seen = c->frames_seen;
+  return ASTRO_OK;
+}
+
+astro_status_t astro_kvcache_set_state(astro_kvcache_t* c, const astro_kvcache_state_t* state) {
+  if (!c || !state) return ASTRO_ERR_NULL;
+  const int S = c->d.sink_frames, L = c->d.window_frames;
+  if (state->sink_held < 0 || state->sink_held > S || state->window_held < 0 || state->window_held > L ||
+      state->window_head < 0 || state->window_head >= L || state->frames_seen < state->sink_held + state->window_held)
+    return ASTRO_ERR_SHAPE;
+  if (state->window_held > 0 && state->sink_held != S) return ASTRO_ERR_SHAPE;  // the sink fills first
+  c->sink_held = state->sink_held;
+  c->win_head = state->window_held == 0 ? 0 : state->window_head;
+  c->win_held = state->window_held;
+  c->frames_seen = state->frames_seen;
+  return ASTRO_OK;
+}
+
 astro_status_t astro_kvcache_export(const astro_kvcache_t* c, void* k_out, void* v_out, void* stream) {
   if (!c || !k_out || !v_out) return ASTRO_ERR_NULL;
   if (!aligned16(k_out) || !aligned16(v_out)) return ASTRO_ERR_ALIGN;

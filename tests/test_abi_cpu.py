@@ -113,3 +113,27 @@ def test_product_never_reaches_the_oracle():
         if f.endswith(".py"):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2603_17051_b200" not in text and "ctypes" not in text, f
+
+
+def test_state_record_round_trip_and_validation():
+    L = A.lib()
+    st, h = _raw_create(A.KVCacheDesc(1, 2, 64, 16, 2, 4))
+    assert st == 0
+    rec = A.KVCacheState()
+    assert L.astro_kvcache_get_state(h, C.byref(rec)) == 0
+    assert (rec.sink_held, rec.window_head, rec.window_held, rec.frames_seen) == (0, 0, 0, 0)
+    good = A.KVCacheState(2, 3, 4, 17)
+    assert L.astro_kvcache_set_state(h, C.byref(good)) == 0
+    assert L.astro_kvcache_get_state(h, C.byref(rec)) == 0
+    assert (rec.sink_held, rec.window_head, rec.window_held, rec.frames_seen) == (2, 3, 4, 17)
+    a, b, c = C.c_int(), C.c_int(), C.c_int64()
+    L.astro_kvcache_query(h, C.byref(a), C.byref(b), C.byref(c))
+    assert (a.value, b.value, c.value) == (2, 4, 17)
+    assert L.astro_kvcache_evict(h, 3, None) == 0                      # ring index advances modulo L
+    L.astro_kvcache_get_state(h, C.byref(rec))
+    assert (rec.window_head, rec.window_held) == (2, 1)
+    for bad in (A.KVCacheState(3, 0, 0, 3), A.KVCacheState(2, 4, 1, 9), A.KVCacheState(2, 0, 5, 9),
+                A.KVCacheState(1, 0, 2, 9), A.KVCacheState(2, 0, 2, 3), A.KVCacheState(-1, 0, 0, 0)):
+        assert L.astro_kvcache_set_state(h, C.byref(bad)) == 2
+    assert L.astro_kvcache_set_state(h, None) == 1
+    L.astro_kvcache_destroy(h)

@@ -86,3 +86,27 @@ def test_append_in_pieces_larger_than_one_launch():
     kb = synth.normal_bf16(8000, (Bc, 42 * T, H, D)); vb = synth.normal_bf16(8001, (Bc, 42 * T, H, D))
     A.astro_kvcache_append(cache, dev_bf16(kb), dev_bf16(vb), 42); model.append(kb, vb, T)
     _both_export_equal(A, cache, model)
+
+
+def test_saved_storage_and_state_resume_on_a_new_handle():
+    """Checkpoint/resume: clone the storage bytes, carry the state record over, continue streaming."""
+    from paper_2603_17051_b200 import binding as A
+    Bc, H, D, T, S, L = 2, 2, 64, 9, 2, 5
+    cache = A.astro_kvcache_create(Bc, H, D, T, S, L)
+    model = orc.RollingKVCache(S, L)
+    seed = 9100
+    for n in range(9):                                       # fill, then churn so the ring head is mid-way
+        if model.held() == S + L:
+            A.astro_kvcache_evict(cache, 2); model.evict(2)
+        kb = synth.normal_bf16(seed, (Bc, T, H, D)); vb = synth.normal_bf16(seed + 1, (Bc, T, H, D)); seed += 2
+        A.astro_kvcache_append(cache, dev_bf16(kb), dev_bf16(vb), 1); model.append(kb, vb, T)
+    state = A.astro_kvcache_get_state(cache)
+    resumed = A.astro_kvcache_create(Bc, H, D, T, S, L, k_storage=cache.k_storage.clone(),
+                                     v_storage=cache.v_storage.clone())
+    A.astro_kvcache_set_state(resumed, state)
+    _both_export_equal(A, resumed, model)
+    A.astro_kvcache_evict(resumed, 1); model.evict(1)
+    kb = synth.normal_bf16(seed, (Bc, T, H, D)); vb = synth.normal_bf16(seed + 1, (Bc, T, H, D))
+    A.astro_kvcache_append(resumed, dev_bf16(kb), dev_bf16(vb), 1); model.append(kb, vb, T)
+    _both_export_equal(A, resumed, model)
+    assert A.astro_kvcache_query(resumed)[2] == model.frames_seen
