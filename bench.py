@@ -433,6 +433,26 @@ def run_extra(args):
                           "config": "B=4 H=12 D=128 T=1560, S=3 + %d window slots, 80 chunks x (evict, 4 fwd, append)" % slots,
                           "frac_of_bf16_sustained": flops / (ms * 1e-3) / 1e12 / peaks["bf16_sustained"]}))
         return 0
+    if args.workload == "nft":
+        # policy loss + selective KL + gradient on the velocity tensors of a 3-frame window (16 x 60 x 104 latents)
+        Bn, E = 96, 3 * 16 * 60 * 104
+        vt, vo, vr, tg = (rnd(30 + i, (Bn, E)) for i in range(4))
+        r = torch.rand(Bn, device=dev); wp = torch.full((Bn,), 1.0 / (Bn * E), device=dev)
+        wk = torch.full((Bn,), 1e-4 / E, device=dev)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        outs = (torch.empty(Bn, device=dev), torch.empty(Bn, device=dev), torch.empty_like(vt))
+        call = lambda: A.astro_nft_loss(vt, vo, vr, tg, r, 1.0, w_policy=wp, w_kl=wk, out=outs)
+        for _ in range(3):
+            call()
+        # 288 MB touched per call (larger than L2); 20 calls back to back so that the device, not the host
+        # submitting two memsets and a kernel per call, sets the pace
+        ms = _event_ms(call, 20)
+        byts = 5 * 2 * Bn * E
+        print(json.dumps({"workload": "nft", "metric": "nft_loss_hbm_gbs", "value": byts / ms / 1e6, "unit": "GB/s",
+                          "ms": ms, "bytes_moved": byts, "config": "96 samples x 299520 elements, 4 bf16 reads + 1 bf16 write, 20 calls back to back",
+                          "roofline": {"bound": "hbm", "achieved": byts / ms / 1e6, "peak": peaks["hbm"], "unit": "GB/s",
+                                       "frac": byts / ms / 1e6 / peaks["hbm"]}}))
+        return 0
     if args.workload == "group":
         # clip-level group-wise sampling: G candidate chunks decode against one frozen, shared prefix
         w = synth.LAYER_FWD
@@ -534,7 +554,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", choices=("layer", "rollout", "rl_update", "sweep", "group"), default="layer",
+    ap.add_argument("--workload", choices=("layer", "rollout", "rl_update", "sweep", "group", "nft"), default="layer",
                     help="layer (default): the contract line; the others print one JSON line per extra workload")
     ap.add_argument("--group", type=int, default=24, help="group workload: candidates G decoding against one prefix")
     ap.add_argument("--replicated", action="store_true",

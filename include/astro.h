@@ -159,6 +159,23 @@ astro_status_t astro_chunk_attn_bwd_dkv(const void* q, const void* k_chunk, cons
                                         int n_q, int n_kc, float scale, void* dk_chunk, void* dv_chunk,
                                         void* stream);
 
+/* Eq. 1, Eq. 2 and the selective KL term of Sec. 3.4 (Algorithm 2, "Policy loss on window"), fused with
+ * the gradient for the current policy, over the velocity tensors of the active window:
+ *   v+ = (1-beta) v_old + beta v_theta;  v- = (1+beta) v_old - beta v_theta;
+ *   policy_i = r_i ||v+ - target||^2 + (1 - r_i) ||v- - target||^2;   kl_i = ||v_theta - v_ref||^2
+ * per sample i, with ||.||^2 the plain sum of squares over the sample's `elems` elements, and
+ *   grad = d/d v_theta of sum_i (w_policy_i policy_i + w_kl_i kl_i)
+ * (the caller folds 1/elems, 1/batch, lambda_KL, the uncertainty mask and 1/|M| into the weights).
+ * v_theta, v_old, v_ref, v_target, grad: device bf16 [batch, elems], 16-byte aligned, elems a multiple of 8.
+ * r_tilde, w_policy, w_kl, policy_out, kl_out: device fp32 [batch].  v_ref and kl_out may be null together
+ * (no KL term); w_policy null means 1, w_kl null means 0; grad may be null (losses only).  policy_out and
+ * kl_out are overwritten.  fp32 arithmetic; the per-sample sums use atomics, so their last bits depend on
+ * the order of the blocks. */
+astro_status_t astro_nft_loss(const void* v_theta, const void* v_old, const void* v_ref, const void* v_target,
+                              const float* r_tilde, const float* w_policy, const float* w_kl, int batch,
+                              long long elems, float beta, float* policy_out, float* kl_out, void* grad,
+                              void* stream);
+
 /* The paper has no counterpart for this call: it exists for callers that must not allocate device
  * memory around the backward -- a training loop whose allocator is frozen after warm-up, a plug-in
  * that runs inside someone else's memory pool, a host thread that may not take the allocator's lock.

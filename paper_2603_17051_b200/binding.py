@@ -16,7 +16,7 @@ STATUS_NAMES = {0: "ASTRO_OK", 1: "ASTRO_ERR_NULL", 2: "ASTRO_ERR_SHAPE", 3: "AS
                 4: "ASTRO_ERR_CAPACITY", 5: "ASTRO_ERR_UNDERFLOW", 6: "ASTRO_ERR_ARCH", 7: "ASTRO_ERR_CUDA",
                 8: "ASTRO_ERR_TIMEOUT"}
 
-EXPORTED = ("astro_kvcache_get_state", "astro_kvcache_set_state", "astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcache_destroy", "astro_kvcache_reset",
+EXPORTED = ("astro_nft_loss", "astro_kvcache_get_state", "astro_kvcache_set_state", "astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcache_destroy", "astro_kvcache_reset",
             "astro_kvcache_append", "astro_kvcache_evict", "astro_kvcache_query", "astro_kvcache_export",
             "astro_chunk_attn_fwd", "astro_chunk_attn_bwd_workspace_bytes", "astro_chunk_attn_bwd",
             "astro_chunk_attn_bwd_delta", "astro_chunk_attn_bwd_dq", "astro_chunk_attn_bwd_dkv",
@@ -86,6 +86,8 @@ def lib():
     L.astro_chunk_attn_bwd_dkv.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp]
     L.astro_chunk_attn_bwd_static.restype = ci
     L.astro_chunk_attn_bwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
+    L.astro_nft_loss.restype = ci
+    L.astro_nft_loss.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, C.c_longlong, cf, vp, vp, vp, vp]
     L.astro_last_device_status.restype = ci
     L.astro_last_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.astro_status_string.restype = C.c_char_p
@@ -292,6 +294,29 @@ def astro_chunk_attn_bwd_dkv(q, k_chunk, v_chunk, lse, delta, d_o, scale: float,
                                         D, n_q, n_kc, float(scale), _ptr(dk_chunk), _ptr(dv_chunk), _stream(stream))
     _check(st, "astro_chunk_attn_bwd_dkv")
     return dk_chunk, dv_chunk
+
+
+def astro_nft_loss(v_theta, v_old, v_ref, v_target, r_tilde, beta: float, w_policy=None, w_kl=None, grad=True,
+                   stream=None, out=None):
+    """Per-sample policy loss and squared distance to the reference, plus d/d v_theta of the weighted total.
+
+    Velocity tensors: bf16 [B, ...] (flattened per sample); r_tilde / weights: fp32 [B].  Returns
+    (policy[B], kl[B] or None, grad like v_theta or None); `out` may pass those three preallocated."""
+    import torch
+    B = v_theta.shape[0]
+    elems = v_theta.numel() // B
+    if out is not None:
+        policy, kl, g = out
+    else:
+        policy = torch.empty(B, dtype=torch.float32, device=v_theta.device)
+        kl = None if v_ref is None else torch.empty(B, dtype=torch.float32, device=v_theta.device)
+        g = torch.empty_like(v_theta) if grad else None
+    for t in (v_theta, v_old, v_ref, v_target):
+        assert t is None or t.is_contiguous()
+    st = lib().astro_nft_loss(_ptr(v_theta), _ptr(v_old), _ptr(v_ref), _ptr(v_target), _ptr(r_tilde), _ptr(w_policy),
+                              _ptr(w_kl), B, elems, float(beta), _ptr(policy), _ptr(kl), _ptr(g), _stream(stream))
+    _check(st, "astro_nft_loss")
+    return policy, kl, g
 
 
 BWD_STATIC_MAX_ROWS = 262144

@@ -12,6 +12,7 @@
 #include "attn_bwd.cuh"
 #include "attn_fwd.cuh"
 #include "kv_ring.cuh"
+#include "nft_loss.cuh"
 
 using namespace astro;
 
@@ -506,6 +507,33 @@ astro_status_t astro_chunk_attn_bwd(const astro_kvcache_t* cache, const void* q,
   if (s != ASTRO_OK || n_kc == 0) return s;
   return astro_chunk_attn_bwd_dkv(q, k_chunk, v_chunk, lse, delta, d_o, batch, heads, head_dim, n_q, n_kc, scale,
                                   dk_chunk, dv_chunk, stream);
+}
+
+astro_status_t astro_nft_loss(const void* v_theta, const void* v_old, const void* v_ref, const void* v_target,
+                              const float* r_tilde, const float* w_policy, const float* w_kl, int batch,
+                              long long elems, float beta, float* policy_out, float* kl_out, void* grad,
+                              void* stream) {
+  if (!v_theta || !v_old || !v_target || !r_tilde || !policy_out) return ASTRO_ERR_NULL;
+  if ((v_ref == nullptr) != (kl_out == nullptr)) return ASTRO_ERR_NULL;
+  if (batch < 1 || batch > 65535 || elems < 8 || (elems & 7)) return ASTRO_ERR_SHAPE;
+  if (!aligned16(v_theta) || !aligned16(v_old) || !aligned16(v_target) || (v_ref && !aligned16(v_ref)) ||
+      (grad && !aligned16(grad)))
+    return ASTRO_ERR_ALIGN;
+  astro_status_t s = check_arch();
+  if (s != ASTRO_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(policy_out, 0, sizeof(float) * batch, st) != cudaSuccess) return ASTRO_ERR_CUDA;
+  if (kl_out && cudaMemsetAsync(kl_out, 0, sizeof(float) * batch, st) != cudaSuccess) return ASTRO_ERR_CUDA;
+  const long long vecs = elems / 8;
+  const long long per_block = static_cast<long long>(kNftThreads) * kNftVecsPerThread;
+  long long blocks = (vecs + per_block - 1) / per_block;
+  if (blocks > 4096) blocks = 4096;
+  dim3 grid(static_cast<unsigned>(blocks), batch);
+  nft_loss_kernel<<<grid, kNftThreads, 0, st>>>(
+      static_cast<const uint4*>(v_theta), static_cast<const uint4*>(v_old), static_cast<const uint4*>(v_ref),
+      static_cast<const uint4*>(v_target), r_tilde, w_policy, w_kl, vecs, beta, policy_out, kl_out,
+      static_cast<uint4*>(grad));
+  return launch_status();
 }
 
 // ---- backward without caller scratch ---------------------------------------------------------------
