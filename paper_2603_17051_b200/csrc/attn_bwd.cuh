@@ -56,11 +56,11 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16* __r
 //   warps 0-3  group 0: keys  0..63  of every key tile (one query row per thread)
 //   warps 4-7  group 1: keys 64..127
 //   warp  8    one thread issues every tcgen05 MMA           warp  9    one thread issues every TMA load
-// Per key tile j the tensor core forms S(j) = Q K^T (two tiles ahead, two buffers) and dP(j) = dO V^T (one
-// buffer), both full 128x128 MMAs.  Each thread exponentiates its 64 S values while the tensor core is busy
-// with the previous tile's dQ and this tile's dP, then turns dP into dS = P o (dP - delta) in place (bf16
-// pairs over its own dP columns) and the tensor core adds dS K into the one dQ accumulator.
-//   TMEM columns: S buffer 0 [0,128)  S buffer 1 [128,256)  dP / dS [256,384)  dQ [384,384+D)
+// Per key tile j: S(j) = Q K^T and dP(j) = dO V^T are full 128x128 MMAs into single buffers that the
+// groups hand back as soon as their values are in registers, so S(j+1) and dP(j+1) are computed while the
+// groups still work on tile j.  dS = P o (dP - delta) goes to one of two bf16 buffers and dQ += dS K
+// follows; no step of tile j+1 waits for the tensor core to finish tile j.
+//   TMEM columns: S [0,128)  dP [128,256)  dS buffer 0 [256,320)  dS buffer 1 [320,384)  dQ [384,384+D)
 constexpr int kDqKStages = 3, kDqVStages = 2;
 constexpr int kDqThreads = 320;
 constexpr int kDqPolyOf8 = 2;  // share of the exponentials evaluated on the FMA pipe
@@ -94,10 +94,12 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   uint64_t* k_empty = k_full + kDqKStages;
   uint64_t* v_full = k_empty + kDqKStages;     // [kDqVStages]
   uint64_t* v_empty = v_full + kDqVStages;
-  uint64_t* s_full = v_empty + kDqVStages;     // [2] per S buffer
-  uint64_t* dp_full = s_full + 2;
-  uint64_t* ds_full = dp_full + 1;             // 256 arrivals: both groups
-  uint64_t* dq_full = ds_full + 1;
+  uint64_t* s_full = v_empty + kDqVStages;     // S(j) computed
+  uint64_t* dp_full = s_full + 1;              // dP(j) computed
+  uint64_t* s_free = dp_full + 1;              // 256 arrivals: every thread has S(j) in registers
+  uint64_t* dp_free = s_free + 1;              // 256 arrivals: every thread has dP(j) in registers
+  uint64_t* ds_full = dp_free + 1;             // [2] per dS buffer, 256 arrivals
+  uint64_t* dq_full = ds_full + 2;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(dq_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
@@ -108,7 +110,7 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   const int h = cache_shared ? blockIdx.z : blockIdx.y, b = cache_shared ? blockIdx.y : blockIdx.z;
   const int bx = cache_shared ? 0 : b;
   constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kColS = 0 /* + 128 * buffer */, kColdP = 256, kColdQ = 384;
+  constexpr uint32_t kColS = 0, kColdP = 128, kColdS = 256 /* + 64 * buffer */, kColdQ = 384;
   constexpr int kMmaWarp = 8, kTmaWarp = 9;
   constexpr int kHalfBytes = 64 * 128;  // 64 rows of a block
   const int n_tiles = seg_tiles(segs);
@@ -118,9 +120,11 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     for (int i = 0; i < kDqKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
     for (int i = 0; i < kDqVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
     mbar_init(s_full, 1);
-    mbar_init(s_full + 1, 1);
     mbar_init(dp_full, 1);
+    mbar_init(s_free, 256);
+    mbar_init(dp_free, 256);
     mbar_init(ds_full, 256);
+    mbar_init(ds_full + 1, 256);
     mbar_init(dq_full, 1);
     *abort_flag = 0;
     fence_mbar_init();
@@ -140,43 +144,30 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       mbar_arrive_expect_tx(q_full, 2 * TileGeom<D>::kBytes);
       tma_load_tile<D>(sQ, &tm_q, q_full, q0, h, b);
       tma_load_tile<D>(sdO, &tm_do, q_full, q0, h, b);
-      // K runs one tile ahead of V: K0 K1 | V0 K2 | V1 K3 | ...  (S is issued two tiles ahead, dP one)
-      KeyTileIter itk, itv;
-      auto load_k = [&](int j) {
-        const int st = j % kDqKStages;
-        const bool fc = itk.from_chunk(segs);
-        mbar_wait_spin(k_empty + st, ((j / kDqKStages) & 1) ^ 1, abort_flag);
-        mbar_arrive_expect_tx(k_full + st, TileGeom<D>::kBytes);
-        tma_load_tile<D>(sK + st * TileGeom<D>::kBytes, fc ? &tm_kc : &tm_kx, k_full + st, itk.row0(segs), h,
+      int j = 0;
+      for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
+        const int sk = j % kDqKStages, sv = j % kDqVStages;
+        const bool fc = it.from_chunk(segs);
+        mbar_wait_spin(k_empty + sk, ((j / kDqKStages) & 1) ^ 1, abort_flag);
+        mbar_arrive_expect_tx(k_full + sk, TileGeom<D>::kBytes);
+        tma_load_tile<D>(sK + sk * TileGeom<D>::kBytes, fc ? &tm_kc : &tm_kx, k_full + sk, it.row0(segs), h,
                          fc ? b : bx);
-        itk.next(segs);
-      };
-      auto load_v = [&](int j) {
-        const int st = j % kDqVStages;
-        const bool fc = itv.from_chunk(segs);
-        mbar_wait_spin(v_empty + st, ((j / kDqVStages) & 1) ^ 1, abort_flag);
-        mbar_arrive_expect_tx(v_full + st, TileGeom<D>::kBytes);
-        tma_load_tile<D>(sV + st * TileGeom<D>::kBytes, fc ? &tm_vc : &tm_vx, v_full + st, itv.row0(segs), h,
+        mbar_wait_spin(v_empty + sv, ((j / kDqVStages) & 1) ^ 1, abort_flag);
+        mbar_arrive_expect_tx(v_full + sv, TileGeom<D>::kBytes);
+        tma_load_tile<D>(sV + sv * TileGeom<D>::kBytes, fc ? &tm_vc : &tm_vx, v_full + sv, it.row0(segs), h,
                          fc ? b : bx);
-        itv.next(segs);
-      };
-      load_k(0);
-      if (n_tiles > 1) load_k(1);
-      for (int j = 0; j < n_tiles; ++j) {
-        load_v(j);
-        if (j + 2 < n_tiles) load_k(j + 2);
       }
     }
   } else if (warp == kMmaWarp) {
     if (lane == 0) {
-      auto issue_s = [&](int j) {  // buffer j & 1 is free: both groups published dS(j-2) after loading S(j-2)
+      auto issue_s = [&](int j) {
         const int st = j % kDqKStages;
         mbar_wait_spin(k_full + st, (j / kDqKStages) & 1, abort_flag);
         tc_fence_after_sync();
-        mma_abT<D>(tmem_base + kColS + (j & 1) * 128, smem_u32(sQ), smem_u32(sK + st * TileGeom<D>::kBytes));
-        mma_commit(s_full + (j & 1));
+        mma_abT<D>(tmem_base + kColS, smem_u32(sQ), smem_u32(sK + st * TileGeom<D>::kBytes));
+        mma_commit(s_full);
       };
-      auto issue_dp = [&](int j) {  // overwrites dS(j-1): issued after the dQ MMAs that read it, MMAs run in order
+      auto issue_dp = [&](int j) {
         const int st = j % kDqVStages;
         mbar_wait_spin(v_full + st, (j / kDqVStages) & 1, abort_flag);
         tc_fence_after_sync();
@@ -187,17 +178,22 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       mbar_wait_spin(q_full, 0, abort_flag);
       issue_s(0);
       issue_dp(0);
-      if (n_tiles > 1) issue_s(1);
       for (int j = 0; j < n_tiles; ++j) {
+        if (j + 1 < n_tiles) {
+          mbar_wait_spin(s_free, j & 1, abort_flag);   // S(j) is in registers everywhere
+          issue_s(j + 1);
+          mbar_wait_spin(dp_free, j & 1, abort_flag);  // dP(j) is in registers everywhere
+          issue_dp(j + 1);
+        }
+        // dS buffer j & 1 was last read by dQ(j-2), issued before S(j) on which this tile's dS depends
         const int st = j % kDqKStages;
         const uint32_t kt = smem_u32(sK + st * TileGeom<D>::kBytes);
-        mbar_wait_spin(ds_full, j & 1, abort_flag);
+        const uint32_t ds = tmem_base + kColdS + (j & 1) * 64;
+        mbar_wait_spin(ds_full + (j & 1), (j >> 1) & 1, abort_flag);
         tc_fence_after_sync();
-        mma_pb<D, 64>(tmem_base + kColdQ, tmem_base + kColdP, kt, j > 0);
-        mma_pb<D, 64>(tmem_base + kColdQ, tmem_base + kColdP + 64, kt + kHalfBytes, true);
+        mma_pb<D, 64>(tmem_base + kColdQ, ds, kt, j > 0);
+        mma_pb<D, 64>(tmem_base + kColdQ, ds + 32, kt + kHalfBytes, true);
         mma_commit(k_empty + st);
-        if (j + 1 < n_tiles) issue_dp(j + 1);
-        if (j + 2 < n_tiles) issue_s(j + 2);
       }
       mma_commit(dq_full);
     }
@@ -216,14 +212,15 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
       const int tile_valid = it.valid(segs);
       const int valid = tile_valid - 64 * g;  // valid keys of this group's half (may be <= 0)
-      const uint32_t colS = kColS + (j & 1) * 128 + g * 64;
-      mbar_wait(s_full + (j & 1), (j >> 1) & 1, abort_flag);
+      mbar_wait(s_full, j & 1, abort_flag);
       tc_fence_after_sync();
       uint32_t s[2][32];
-      tmem_ld32(tmem_lane + colS, s[0]);
-      tmem_ld32(tmem_lane + colS + 32, s[1]);
+      tmem_ld32(tmem_lane + kColS + g * 64, s[0]);
+      tmem_ld32(tmem_lane + kColS + g * 64 + 32, s[1]);
       tmem_wait_ld();
-      // P = exp2(s * scale * log2e - LSE * log2e), kept as packed fp32 pairs in the registers of S
+      tc_fence_before_sync();
+      mbar_arrive(s_free);
+      // P = exp2(s * scale * log2e - LSE * log2e), kept as packed fp32 pairs
       uint64_t p2[2][16];
 #pragma unroll
       for (int c2 = 0; c2 < 2; ++c2)
@@ -243,33 +240,33 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
       mbar_wait(dp_full, j & 1, abort_flag);
       tc_fence_after_sync();
+      uint32_t dp[2][32], ds[32];
+      tmem_ld32(tmem_lane + kColdP + g * 64, dp[0]);
+      tmem_ld32(tmem_lane + kColdP + g * 64 + 32, dp[1]);
+      tmem_wait_ld();
+      tc_fence_before_sync();
+      mbar_arrive(dp_free);
 #pragma unroll
-      for (int c2 = 0; c2 < 2; ++c2) {
-        uint32_t dp[32], ds[16];
-        tmem_ld32(tmem_lane + kColdP + g * 64 + c2 * 32, dp);
-        tmem_wait_ld();
+      for (int c2 = 0; c2 < 2; ++c2)
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
           const uint64_t d2 = mul2(p2[c2][c >> 1],
-                                   add2(f32x2(__uint_as_float(dp[c]), __uint_as_float(dp[c + 1])), nd2));
+                                   add2(f32x2(__uint_as_float(dp[c2][c]), __uint_as_float(dp[c2][c + 1])), nd2));
           float d0, d1;
           f32x2_split(d2, d0, d1);
           if (valid < 64) {  // stale keys past the segment's end: S and dP hold anything, dS must be 0
             if (c2 * 32 + c >= valid) d0 = 0.f;
             if (c2 * 32 + c + 1 >= valid) d1 = 0.f;
           }
-          ds[c >> 1] = pack_bf16(d0, d1);
+          ds[c2 * 16 + (c >> 1)] = pack_bf16(d0, d1);
         }
-        // in place: the 16 packed columns written here lie inside the 32 dP columns just read (c2 = 0) or
-        // inside columns read one step earlier (c2 = 1), all owned by this thread
-        tmem_st16(tmem_lane + kColdP + g * 64 + c2 * 16, ds);
-      }
+      tmem_st32(tmem_lane + kColdS + (j & 1) * 64 + g * 32, ds);
       // Key rows past the segment's end may hold stale cache contents: dS is 0 there, but 0 * NaN is NaN.
       if (g == 0 && tile_valid < kTile)
         zero_tile_rows_from<D>(sK + (j % kDqKStages) * TileGeom<D>::kBytes, tile_valid, r);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(ds_full);
+      mbar_arrive(ds_full + (j & 1));
     }
     // ---- epilogue: group g writes columns [g D/2, (g+1) D/2) of dQ
     mbar_wait(dq_full, 0, abort_flag);
