@@ -171,7 +171,7 @@ astro_status_t check_attn_args(const AttnArgs& a, float scale) {
 }
 
 template <int D>
-astro_status_t launch_fwd(const AttnArgs& a, const CUtensorMap& tq, const CUtensorMap& tkc, const CUtensorMap& tvc,
+astro_status_t launch_fwd(const AttnArgs& a, const __nv_bfloat16* q, const CUtensorMap& tkc, const CUtensorMap& tvc,
                           const CUtensorMap& tkx, const CUtensorMap& tvx, const KeySegs& segs, float scale, void* o,
                           float* lse, cudaStream_t st) {
   static bool done[64];
@@ -180,7 +180,7 @@ astro_status_t launch_fwd(const AttnArgs& a, const CUtensorMap& tq, const CUtens
   const int shared = (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
   dim3 grid((a.n_q + kTile - 1) / kTile, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
   chunk_attn_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kTotal, st>>>(
-      tq, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared,
+      q, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared,
       scale * kLog2e, static_cast<__nv_bfloat16*>(o), lse);
   return launch_status();
 }
@@ -391,10 +391,9 @@ astro_status_t astro_chunk_attn_fwd(const astro_kvcache_t* cache, const void* q,
   s = check_arch();
   if (s != ASTRO_OK) return s;
   const bool have_ctx = cache && (cache->sink_held + cache->win_held) > 0;
-  CUtensorMap tq, tkc, tvc, tkx, tvx;
+  CUtensorMap tkc, tvc, tkx, tvx;
   std::memset(&tkc, 0, sizeof(tkc)); std::memset(&tvc, 0, sizeof(tvc));
   std::memset(&tkx, 0, sizeof(tkx)); std::memset(&tvx, 0, sizeof(tvx));
-  if ((s = make_tmap_user(&tq, q, head_dim, n_q, heads, batch)) != ASTRO_OK) return s;
   if (n_kc > 0) {
     if ((s = make_tmap_user(&tkc, k_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
     if ((s = make_tmap_user(&tvc, v_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
@@ -406,8 +405,9 @@ astro_status_t astro_chunk_attn_fwd(const astro_kvcache_t* cache, const void* q,
   }
   const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return head_dim == 128 ? launch_fwd<128>(a, tq, tkc, tvc, tkx, tvx, segs, scale, o, lse, st)
-                         : launch_fwd<64>(a, tq, tkc, tvc, tkx, tvx, segs, scale, o, lse, st);
+  const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q);
+  return head_dim == 128 ? launch_fwd<128>(a, qp, tkc, tvc, tkx, tvx, segs, scale, o, lse, st)
+                         : launch_fwd<64>(a, qp, tkc, tvc, tkx, tvx, segs, scale, o, lse, st);
 }
 
 size_t astro_chunk_attn_bwd_workspace_bytes(int batch, int heads, int n_q, int head_dim) {

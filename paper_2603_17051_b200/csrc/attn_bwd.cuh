@@ -53,16 +53,18 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16* __r
 
 // ------------------------------------------------------------------------------------------ dQ
 // Warp-specialised, one CTA (one 128-query tile) per SM:
-//   warps 0-3  group 0: keys  0..63  of every key tile (one query row per thread)
-//   warps 4-7  group 1: keys 64..127
-//   warp  8    one thread issues every tcgen05 MMA           warp  9    one thread issues every TMA load
+//   kDqGroups groups of 4 warps; group g owns keys [g, g+1) * 128 / kDqGroups of every key tile, one query
+//   row per thread; then one warp whose first thread issues every tcgen05 MMA and one for every TMA load
 // Per key tile j: S(j) = Q K^T and dP(j) = dO V^T are full 128x128 MMAs into single buffers that the
 // groups hand back as soon as their values are in registers, so S(j+1) and dP(j+1) are computed while the
 // groups still work on tile j.  dS = P o (dP - delta) goes to one of two bf16 buffers and dQ += dS K
 // follows; no step of tile j+1 waits for the tensor core to finish tile j.
 //   TMEM columns: S [0,128)  dP [128,256)  dS buffer 0 [256,320)  dS buffer 1 [320,384)  dQ [384,384+D)
 constexpr int kDqKStages = 3, kDqVStages = 2;
-constexpr int kDqThreads = 320;
+constexpr int kDqGroups = 2;                      // softmax groups: more warps per scheduler hide the
+constexpr int kDqCols = kTile / kDqGroups;         // exp2 latency behind the arithmetic of the other warps
+constexpr int kDqSoftmaxThreads = 128 * kDqGroups;
+constexpr int kDqThreads = kDqSoftmaxThreads + 64;
 constexpr int kDqPolyOf8 = 2;  // share of the exponentials evaluated on the FMA pipe
 
 template <int D> struct DqSmem {
@@ -111,7 +113,7 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   const int bx = cache_shared ? 0 : b;
   constexpr uint32_t kTmemCols = 512;
   constexpr uint32_t kColS = 0, kColdP = 128, kColdS = 256 /* + 64 * buffer */, kColdQ = 384;
-  constexpr int kMmaWarp = 8, kTmaWarp = 9;
+  constexpr int kMmaWarp = 4 * kDqGroups, kTmaWarp = 4 * kDqGroups + 1;
   constexpr int kHalfBytes = 64 * 128;  // 64 rows of a block
   const int n_tiles = seg_tiles(segs);
 
@@ -121,10 +123,10 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     for (int i = 0; i < kDqVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
     mbar_init(s_full, 1);
     mbar_init(dp_full, 1);
-    mbar_init(s_free, 256);
-    mbar_init(dp_free, 256);
-    mbar_init(ds_full, 256);
-    mbar_init(ds_full + 1, 256);
+    mbar_init(s_free, kDqSoftmaxThreads);
+    mbar_init(dp_free, kDqSoftmaxThreads);
+    mbar_init(ds_full, kDqSoftmaxThreads);
+    mbar_init(ds_full + 1, kDqSoftmaxThreads);
     mbar_init(dq_full, 1);
     *abort_flag = 0;
     fence_mbar_init();
@@ -211,19 +213,20 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     int j = 0;
     for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
       const int tile_valid = it.valid(segs);
-      const int valid = tile_valid - 64 * g;  // valid keys of this group's half (may be <= 0)
+      const int valid = tile_valid - kDqCols * g;  // valid keys of this group's share (may be <= 0)
       mbar_wait(s_full, j & 1, abort_flag);
       tc_fence_after_sync();
-      uint32_t s[2][32];
-      tmem_ld32(tmem_lane + kColS + g * 64, s[0]);
-      tmem_ld32(tmem_lane + kColS + g * 64 + 32, s[1]);
+      constexpr int NL = kDqCols / 32;
+      uint32_t s[NL][32];
+#pragma unroll
+      for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + kColS + g * kDqCols + c2 * 32, s[c2]);
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(s_free);
       // P = exp2(s * scale * log2e - LSE * log2e), kept as packed fp32 pairs
-      uint64_t p2[2][16];
+      uint64_t p2[NL][16];
 #pragma unroll
-      for (int c2 = 0; c2 < 2; ++c2)
+      for (int c2 = 0; c2 < NL; ++c2)
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
           const uint64_t x2 = fma2(f32x2(__uint_as_float(s[c2][c]), __uint_as_float(s[c2][c + 1])), sc2, nl2);
@@ -240,27 +243,29 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
       mbar_wait(dp_full, j & 1, abort_flag);
       tc_fence_after_sync();
-      uint32_t dp[2][32], ds[32];
-      tmem_ld32(tmem_lane + kColdP + g * 64, dp[0]);
-      tmem_ld32(tmem_lane + kColdP + g * 64 + 32, dp[1]);
+      uint32_t dp[NL][32], ds[NL][16];
+#pragma unroll
+      for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + kColdP + g * kDqCols + c2 * 32, dp[c2]);
       tmem_wait_ld();
       tc_fence_before_sync();
       mbar_arrive(dp_free);
 #pragma unroll
-      for (int c2 = 0; c2 < 2; ++c2)
+      for (int c2 = 0; c2 < NL; ++c2)
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
           const uint64_t d2 = mul2(p2[c2][c >> 1],
                                    add2(f32x2(__uint_as_float(dp[c2][c]), __uint_as_float(dp[c2][c + 1])), nd2));
           float d0, d1;
           f32x2_split(d2, d0, d1);
-          if (valid < 64) {  // stale keys past the segment's end: S and dP hold anything, dS must be 0
+          if (valid < kDqCols) {  // stale keys past the segment's end: S and dP hold anything, dS must be 0
             if (c2 * 32 + c >= valid) d0 = 0.f;
             if (c2 * 32 + c + 1 >= valid) d1 = 0.f;
           }
-          ds[c2 * 16 + (c >> 1)] = pack_bf16(d0, d1);
+          ds[c2][c >> 1] = pack_bf16(d0, d1);
         }
-      tmem_st32(tmem_lane + kColdS + (j & 1) * 64 + g * 32, ds);
+#pragma unroll
+      for (int c2 = 0; c2 < NL; ++c2)
+        tmem_st16(tmem_lane + kColdS + (j & 1) * 64 + g * (kDqCols / 2) + c2 * 16, ds[c2]);
       // Key rows past the segment's end may hold stale cache contents: dS is 0 there, but 0 * NaN is NaN.
       if (g == 0 && tile_valid < kTile)
         zero_tile_rows_from<D>(sK + (j % kDqKStages) * TileGeom<D>::kBytes, tile_valid, r);
@@ -268,11 +273,13 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
       tc_fence_before_sync();
       mbar_arrive(ds_full + (j & 1));
     }
-    // ---- epilogue: group g writes columns [g D/2, (g+1) D/2) of dQ
+    // ---- epilogue: groups 0 and 1 write columns [g D/2, (g+1) D/2) of dQ
     mbar_wait(dq_full, 0, abort_flag);
     tc_fence_after_sync();
-    __nv_bfloat16* dst = dq + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + g * (D / 2);
-    store_row_from_tmem<D / 2>(tmem_lane + kColdQ + g * (D / 2), scale, dst, in_range);
+    if (g < 2) {
+      __nv_bfloat16* dst = dq + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + g * (D / 2);
+      store_row_from_tmem<D / 2>(tmem_lane + kColdQ + g * (D / 2), scale, dst, in_range);
+    }
   }
 
   tc_fence_before_sync();

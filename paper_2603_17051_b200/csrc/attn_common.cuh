@@ -52,16 +52,25 @@ __device__ __forceinline__ void tma_load_tile(uint8_t* smem_tile, const CUtensor
     tma_load_4d(smem_tile + blk * TileGeom<D>::kBlockBytes, tm, bar, blk * 64, row0, h, b);
 }
 
-// acc[128 x N] = A[128 x D] * B[N x D]^T, both tiles K-major (contraction over D).  B may start at any
-// multiple of 8 rows inside a 128-row tile (b_smem + rows * 128).
+// The single MMA-issuing thread is latency bound on scalar work, so descriptors are built once per tile
+// operand and stepped by adding to the start-address field (bits 0-13, units of 16 bytes; tiles live below
+// 256 KB, so the field never overflows into its neighbours).
+__device__ __forceinline__ uint64_t desc_step(uint64_t desc, uint32_t byte_offset) { return desc + (byte_offset >> 4); }
+
+// acc[128 x N] = A[128 x D] * B[N x D]^T, both tiles K-major (contraction over D), given the descriptors of
+// the tiles' first bytes.  B may start at any multiple of 8 rows inside a 128-row tile (+ rows * 128 bytes).
 template <int D, int N = kTile>
-__device__ __forceinline__ void mma_abT(uint32_t d_tmem, uint32_t a_smem, uint32_t b_smem) {
+__device__ __forceinline__ void mma_abT_desc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc) {
   constexpr uint32_t idesc = make_idesc_bf16(kTile, N, false, false);
 #pragma unroll
   for (int k = 0; k < D / 16; ++k) {
     const uint32_t off = (k >> 2) * TileGeom<D>::kBlockBytes + (k & 3) * 32;
-    mma_ss(d_tmem, desc_kmajor(a_smem + off), desc_kmajor(b_smem + off), idesc, k > 0);
+    mma_ss(d_tmem, desc_step(a_desc, off), desc_step(b_desc, off), idesc, k > 0);
   }
+}
+template <int D, int N = kTile>
+__device__ __forceinline__ void mma_abT(uint32_t d_tmem, uint32_t a_smem, uint32_t b_smem) {
+  mma_abT_desc<D, N>(d_tmem, desc_kmajor(a_smem), desc_kmajor(b_smem));
 }
 
 // acc[128 x D] (+)= A_tmem[128 x KROWS bf16] * B[KROWS x D] with the contraction over B's rows (MN-major
@@ -69,10 +78,10 @@ __device__ __forceinline__ void mma_abT(uint32_t d_tmem, uint32_t a_smem, uint32
 template <int D, int KROWS = kTile>
 __device__ __forceinline__ void mma_pb(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_smem, bool accumulate) {
   constexpr uint32_t idesc = make_idesc_bf16(kTile, D, false, true);
+  const uint64_t b_desc = desc_mnmajor(b_smem, TileGeom<D>::kBlockBytes);
 #pragma unroll
   for (int k = 0; k < KROWS / 16; ++k)
-    mma_ts(d_tmem, a_tmem + k * 8, desc_mnmajor(b_smem + k * 2048, TileGeom<D>::kBlockBytes), idesc,
-           (accumulate || k > 0) ? 1u : 0u);
+    mma_ts(d_tmem, a_tmem + k * 8, desc_step(b_desc, k * 2048), idesc, (accumulate || k > 0) ? 1u : 0u);
 }
 
 // Zero rows [first_row, 128) of a tile in shared memory (every block), then publish to the async proxy.
