@@ -196,7 +196,7 @@ astro_status_t launch_bwd_delta(const void* o, const void* d_o, int batch, int h
 }
 
 template <int D>
-astro_status_t launch_bwd_dq(const AttnArgs& a, const CUtensorMap& tq, const CUtensorMap& tdo, const CUtensorMap& tkc,
+astro_status_t launch_bwd_dq(const AttnArgs& a, const __nv_bfloat16* q, const CUtensorMap& tdo, const CUtensorMap& tkc,
                              const CUtensorMap& tvc, const CUtensorMap& tkx, const CUtensorMap& tvx,
                              const KeySegs& segs, float scale, const float* lse, const float* delta, void* dq,
                              cudaStream_t st) {
@@ -206,7 +206,7 @@ astro_status_t launch_bwd_dq(const AttnArgs& a, const CUtensorMap& tq, const CUt
   const int shared = (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
   dim3 grid_q((a.n_q + kTile - 1) / kTile, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
   chunk_attn_bwd_dq_kernel<D><<<grid_q, kDqThreads, DqSmem<D>::kTotal, st>>>(
-      tq, tdo, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared, scale, lse, delta,
+      q, tdo, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared, scale, lse, delta,
       static_cast<__nv_bfloat16*>(dq));
   return launch_status();
 }
@@ -443,10 +443,9 @@ astro_status_t astro_chunk_attn_bwd_dq(const astro_kvcache_t* cache, const void*
   s = check_arch();
   if (s != ASTRO_OK) return s;
   const bool have_ctx = cache && (cache->sink_held + cache->win_held) > 0;
-  CUtensorMap tq, tdo, tkc, tvc, tkx, tvx;
+  CUtensorMap tdo, tkc, tvc, tkx, tvx;
   std::memset(&tkc, 0, sizeof(tkc)); std::memset(&tvc, 0, sizeof(tvc));
   std::memset(&tkx, 0, sizeof(tkx)); std::memset(&tvx, 0, sizeof(tvx));
-  if ((s = make_tmap_user(&tq, q, head_dim, n_q, heads, batch)) != ASTRO_OK) return s;
   if ((s = make_tmap_user(&tdo, d_o, head_dim, n_q, heads, batch)) != ASTRO_OK) return s;
   if (n_kc > 0) {
     if ((s = make_tmap_user(&tkc, k_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
@@ -459,8 +458,9 @@ astro_status_t astro_chunk_attn_bwd_dq(const astro_kvcache_t* cache, const void*
   }
   const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return head_dim == 128 ? launch_bwd_dq<128>(a, tq, tdo, tkc, tvc, tkx, tvx, segs, scale, lse, delta, dq, st)
-                         : launch_bwd_dq<64>(a, tq, tdo, tkc, tvc, tkx, tvx, segs, scale, lse, delta, dq, st);
+  const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q);
+  return head_dim == 128 ? launch_bwd_dq<128>(a, qp, tdo, tkc, tvc, tkx, tvx, segs, scale, lse, delta, dq, st)
+                         : launch_bwd_dq<64>(a, qp, tdo, tkc, tvc, tkx, tvx, segs, scale, lse, delta, dq, st);
 }
 
 astro_status_t astro_chunk_attn_bwd_dkv(const void* q, const void* k_chunk, const void* v_chunk, const float* lse,

@@ -57,9 +57,10 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16* __r
 //   row per thread; then one warp whose first thread issues every tcgen05 MMA and one for every TMA load
 // Per key tile j: S(j) = Q K^T and dP(j) = dO V^T are full 128x128 MMAs into single buffers that the
 // groups hand back as soon as their values are in registers, so S(j+1) and dP(j+1) are computed while the
-// groups still work on tile j.  dS = P o (dP - delta) goes to one of two bf16 buffers and dQ += dS K
-// follows; no step of tile j+1 waits for the tensor core to finish tile j.
-//   TMEM columns: S [0,128)  dP [128,256)  dS buffer 0 [256,320)  dS buffer 1 [320,384)  dQ [384,384+D)
+// groups still work on tile j.  dS = P o (dP - delta) goes to a bf16 buffer and dQ += dS K follows.  Q lives
+// in tensor memory (bf16 pairs, written once by the softmax threads) as the A operand of S, which takes a
+// quarter of the operand traffic off shared memory.
+//   TMEM columns: S [0,128)  dP [128,256)  dS [256,320)  Q [320,320+D/2)  dQ [384,384+D)
 constexpr int kDqKStages = 3, kDqVStages = 2;
 constexpr int kDqGroups = 2;                      // softmax groups: more warps per scheduler hide the
 constexpr int kDqCols = kTile / kDqGroups;         // exp2 latency behind the arithmetic of the other warps
@@ -68,9 +69,8 @@ constexpr int kDqThreads = kDqSoftmaxThreads + 64;
 constexpr int kDqPolyOf8 = 2;  // share of the exponentials evaluated on the FMA pipe
 
 template <int D> struct DqSmem {
-  static constexpr int kQ = 0;
-  static constexpr int kdO = TileGeom<D>::kBytes;
-  static constexpr int kK = 2 * TileGeom<D>::kBytes;
+  static constexpr int kdO = 0;
+  static constexpr int kK = TileGeom<D>::kBytes;
   static constexpr int kV = kK + kDqKStages * TileGeom<D>::kBytes;
   static constexpr int kBars = kV + kDqVStages * TileGeom<D>::kBytes;
   static constexpr int kTotal = kBars + 256 + 1024;
@@ -78,7 +78,7 @@ template <int D> struct DqSmem {
 
 template <int D>
 __global__ void __launch_bounds__(kDqThreads, 1)
-chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
+chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant__ CUtensorMap tm_do,
                          const __grid_constant__ CUtensorMap tm_kc, const __grid_constant__ CUtensorMap tm_vc,
                          const __grid_constant__ CUtensorMap tm_kx, const __grid_constant__ CUtensorMap tm_vx,
                          const KeySegs segs, const int n_q, const int heads, const int cache_shared,
@@ -86,7 +86,6 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                          __nv_bfloat16* __restrict__ dq) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
-  uint8_t* sQ = smem + DqSmem<D>::kQ;
   uint8_t* sdO = smem + DqSmem<D>::kdO;
   uint8_t* sK = smem + DqSmem<D>::kK;
   uint8_t* sV = smem + DqSmem<D>::kV;
@@ -100,8 +99,10 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   uint64_t* dp_full = s_full + 1;              // dP(j) computed
   uint64_t* s_free = dp_full + 1;              // 256 arrivals: every thread has S(j) in registers
   uint64_t* dp_free = s_free + 1;              // 256 arrivals: every thread has dP(j) in registers
-  uint64_t* ds_full = dp_free + 1;             // [2] per dS buffer, 256 arrivals
-  uint64_t* dq_full = ds_full + 2;
+  uint64_t* ds_full = dp_free + 1;             // every thread has written its part of dS(j)
+  uint64_t* dq_done = ds_full + 1;             // dQ(j) has consumed dS(j)
+  uint64_t* qt_full = dq_done + 1;             // Q is in tensor memory
+  uint64_t* dq_full = qt_full + 1;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(dq_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
@@ -112,7 +113,7 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
   const int h = cache_shared ? blockIdx.z : blockIdx.y, b = cache_shared ? blockIdx.y : blockIdx.z;
   const int bx = cache_shared ? 0 : b;
   constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kColS = 0, kColdP = 128, kColdS = 256 /* + 64 * buffer */, kColdQ = 384;
+  constexpr uint32_t kColS = 0, kColdP = 128, kColdS = 256, kColQ = 320, kColdQ = 384;
   constexpr int kMmaWarp = 4 * kDqGroups, kTmaWarp = 4 * kDqGroups + 1;
   constexpr int kHalfBytes = 64 * 128;  // 64 rows of a block
   const int n_tiles = seg_tiles(segs);
@@ -126,7 +127,8 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     mbar_init(s_free, kDqSoftmaxThreads);
     mbar_init(dp_free, kDqSoftmaxThreads);
     mbar_init(ds_full, kDqSoftmaxThreads);
-    mbar_init(ds_full + 1, kDqSoftmaxThreads);
+    mbar_init(dq_done, 1);
+    mbar_init(qt_full, 128 * (D / 64));
     mbar_init(dq_full, 1);
     *abort_flag = 0;
     fence_mbar_init();
@@ -143,8 +145,7 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 
   if (warp == kTmaWarp) {
     if (lane == 0) {
-      mbar_arrive_expect_tx(q_full, 2 * TileGeom<D>::kBytes);
-      tma_load_tile<D>(sQ, &tm_q, q_full, q0, h, b);
+      mbar_arrive_expect_tx(q_full, TileGeom<D>::kBytes);
       tma_load_tile<D>(sdO, &tm_do, q_full, q0, h, b);
       int j = 0;
       for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
@@ -162,11 +163,17 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     }
   } else if (warp == kMmaWarp) {
     if (lane == 0) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kTile, false, false);
+      const uint64_t k_desc0 = desc_kmajor(smem_u32(sK));
       auto issue_s = [&](int j) {
         const int st = j % kDqKStages;
         mbar_wait_spin(k_full + st, (j / kDqKStages) & 1, abort_flag);
         tc_fence_after_sync();
-        mma_abT<D>(tmem_base + kColS, smem_u32(sQ), smem_u32(sK + st * TileGeom<D>::kBytes));
+        const uint64_t k_desc = desc_step(k_desc0, st * TileGeom<D>::kBytes);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)  // 16 elements of the head dimension = 8 packed Q columns
+          mma_ts(tmem_base + kColS, tmem_base + kColQ + k * 8,
+                 desc_step(k_desc, (k >> 2) * TileGeom<D>::kBlockBytes + (k & 3) * 32), idesc_s, k > 0);
         mma_commit(s_full);
       };
       auto issue_dp = [&](int j) {
@@ -177,7 +184,9 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         mma_commit(v_empty + st);
         mma_commit(dp_full);
       };
+      mbar_wait_spin(qt_full, 0, abort_flag);
       mbar_wait_spin(q_full, 0, abort_flag);
+      tc_fence_after_sync();
       issue_s(0);
       issue_dp(0);
       for (int j = 0; j < n_tiles; ++j) {
@@ -187,15 +196,13 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
           mbar_wait_spin(dp_free, j & 1, abort_flag);  // dP(j) is in registers everywhere
           issue_dp(j + 1);
         }
-        // dS buffer j & 1 was last read by dQ(j-2), issued before S(j) on which this tile's dS depends
         const int st = j % kDqKStages;
         const uint32_t kt = smem_u32(sK + st * TileGeom<D>::kBytes);
-        const uint32_t ds = tmem_base + kColdS + (j & 1) * 64;
-        mbar_wait_spin(ds_full + (j & 1), (j >> 1) & 1, abort_flag);
+        mbar_wait_spin(ds_full, j & 1, abort_flag);
         tc_fence_after_sync();
-        mma_pb<D, 64>(tmem_base + kColdQ, ds, kt, j > 0);
-        mma_pb<D, 64>(tmem_base + kColdQ, ds + 32, kt + kHalfBytes, true);
+        mma_pb<D, kTile>(tmem_base + kColdQ, tmem_base + kColdS, kt, j > 0);
         mma_commit(k_empty + st);
+        mma_commit(dq_done);
       }
       mma_commit(dq_full);
     }
@@ -210,6 +217,20 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const float delta_r = in_range ? delta[stat_idx] : 0.f;
     const float scale_log2 = scale * kLog2e;
     const uint64_t sc2 = f32x2(scale_log2, scale_log2), nl2 = f32x2(-lse2, -lse2), nd2 = f32x2(-delta_r, -delta_r);
+    // Q row -> tensor memory: group g writes elements [64g, 64g+64) of its row as 32 packed columns
+    if (g * 64 < D) {
+      uint32_t qr[32];
+      const uint4* src = reinterpret_cast<const uint4*>(q + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + g * 64);
+#pragma unroll
+      for (int v = 0; v < 8; ++v) {
+        const uint4 t = in_range ? src[v] : make_uint4(0, 0, 0, 0);
+        qr[4 * v] = t.x; qr[4 * v + 1] = t.y; qr[4 * v + 2] = t.z; qr[4 * v + 3] = t.w;
+      }
+      tmem_st32(tmem_lane + kColQ + g * 32, qr);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(qt_full);
+    }
     int j = 0;
     for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
       const int tile_valid = it.valid(segs);
@@ -263,15 +284,19 @@ chunk_attn_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
           }
           ds[c2][c >> 1] = pack_bf16(d0, d1);
         }
+      if (j > 0) {  // the one dS buffer is free once dQ(j-1) has consumed it (almost always long since)
+        mbar_wait(dq_done, (j - 1) & 1, abort_flag);
+        tc_fence_after_sync();
+      }
 #pragma unroll
       for (int c2 = 0; c2 < NL; ++c2)
-        tmem_st16(tmem_lane + kColdS + (j & 1) * 64 + g * (kDqCols / 2) + c2 * 16, ds[c2]);
+        tmem_st16(tmem_lane + kColdS + g * (kDqCols / 2) + c2 * 16, ds[c2]);
       // Key rows past the segment's end may hold stale cache contents: dS is 0 there, but 0 * NaN is NaN.
       if (g == 0 && tile_valid < kTile)
         zero_tile_rows_from<D>(sK + (j % kDqKStages) * TileGeom<D>::kBytes, tile_valid, r);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(ds_full + (j & 1));
+      mbar_arrive(ds_full);
     }
     // ---- epilogue: groups 0 and 1 write columns [g D/2, (g+1) D/2) of dQ
     mbar_wait(dq_full, 0, abort_flag);
