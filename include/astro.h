@@ -202,6 +202,12 @@ astro_status_t astro_chunk_attn_bwd_static(const astro_kvcache_t* cache, const v
  * (then *detail, a HOST pointer that may be null, receives the raw word). */
 astro_status_t astro_last_device_status(uint32_t* detail);
 
+/* Self-test of that mechanism (the paper has no counterpart): enqueues a one-warp kernel that waits about a
+ * millisecond on a barrier nothing will ever complete.  The kernel gives up, ends normally and leaves the
+ * time-out in the status word, so the next astro_last_device_status returns ASTRO_ERR_TIMEOUT and the
+ * context stays usable.  Nothing faults or hangs. */
+astro_status_t astro_selftest_wait_timeout(void* stream);
+
 /* Static, never null. */
 const char* astro_status_string(astro_status_t status);
 

@@ -16,7 +16,7 @@ STATUS_NAMES = {0: "ASTRO_OK", 1: "ASTRO_ERR_NULL", 2: "ASTRO_ERR_SHAPE", 3: "AS
                 4: "ASTRO_ERR_CAPACITY", 5: "ASTRO_ERR_UNDERFLOW", 6: "ASTRO_ERR_ARCH", 7: "ASTRO_ERR_CUDA",
                 8: "ASTRO_ERR_TIMEOUT"}
 
-EXPORTED = ("astro_nft_loss", "astro_kvcache_get_state", "astro_kvcache_set_state", "astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcache_destroy", "astro_kvcache_reset",
+EXPORTED = ("astro_selftest_wait_timeout", "astro_nft_loss", "astro_kvcache_get_state", "astro_kvcache_set_state", "astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcache_destroy", "astro_kvcache_reset",
             "astro_kvcache_append", "astro_kvcache_evict", "astro_kvcache_query", "astro_kvcache_export",
             "astro_chunk_attn_fwd", "astro_chunk_attn_bwd_workspace_bytes", "astro_chunk_attn_bwd",
             "astro_chunk_attn_bwd_delta", "astro_chunk_attn_bwd_dq", "astro_chunk_attn_bwd_dkv",
@@ -88,6 +88,8 @@ def lib():
     L.astro_chunk_attn_bwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
     L.astro_nft_loss.restype = ci
     L.astro_nft_loss.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, C.c_longlong, cf, vp, vp, vp, vp]
+    L.astro_selftest_wait_timeout.restype = ci
+    L.astro_selftest_wait_timeout.argtypes = [vp]
     L.astro_last_device_status.restype = ci
     L.astro_last_device_status.argtypes = [C.POINTER(C.c_uint32)]
     L.astro_status_string.restype = C.c_char_p
@@ -335,6 +337,11 @@ def astro_chunk_attn_bwd_static(cache, q, k_chunk, v_chunk, o, lse, d_o, scale: 
                                            float(scale), _ptr(dq), _ptr(dk_chunk), _ptr(dv_chunk), _stream(stream))
     _check(st, "astro_chunk_attn_bwd_static")
     return dq, dk_chunk, dv_chunk
+
+
+def astro_selftest_wait_timeout(stream=None) -> None:
+    """Enqueue the bounded-wait self-test kernel (its wait runs out on purpose; see astro_last_device_status)."""
+    _check(lib().astro_selftest_wait_timeout(_stream(stream)), "astro_selftest_wait_timeout")
 
 
 def astro_last_device_status() -> int:

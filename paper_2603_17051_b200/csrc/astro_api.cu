@@ -28,6 +28,23 @@ struct astro_kvcache {
   CUtensorMap tm_k, tm_v;
 };
 
+namespace astro {
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing will ever complete.  The wait
+// gives up after `cycle_limit` clocks, records the time-out in the device status word and the kernel ends
+// normally, which is exactly the path a broken hand-off in the attention kernels would take.
+__global__ void wait_timeout_selftest_kernel(long long cycle_limit) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  mbar_wait_spin(&bar, 0, &abort_flag, cycle_limit);
+}
+}  // namespace astro
+
 namespace {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -577,6 +594,13 @@ astro_status_t astro_chunk_attn_bwd_static(const astro_kvcache_t* cache, const v
   if (s != ASTRO_OK || n_kc == 0) return s;
   return astro_chunk_attn_bwd_dkv(q, k_chunk, v_chunk, lse, delta, d_o, batch, heads, head_dim, n_q, n_kc, scale,
                                   dk_chunk, dv_chunk, stream);
+}
+
+astro_status_t astro_selftest_wait_timeout(void* stream) {
+  astro_status_t s = check_arch();
+  if (s != ASTRO_OK) return s;
+  wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(2000000LL);  // about 1 ms
+  return launch_status();
 }
 
 astro_status_t astro_last_device_status(uint32_t* detail) {

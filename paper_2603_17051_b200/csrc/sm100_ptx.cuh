@@ -56,7 +56,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // releasing its tensor memory.
 constexpr long long kWaitCycleLimit = 400LL * 1000 * 1000;  // about 0.2 s at ~2 GHz
 
-__device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                               long long cycle_limit = kWaitCycleLimit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t it = 0;
@@ -64,7 +65,7 @@ __device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, v
     if (mbar_try_wait(bar, parity)) return true;
     if ((++it & 63u) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycleLimit) {
+      if (clock64() - t0 > cycle_limit) {
         *abort_flag = 1;
         atomicOr(&g_device_status, kStatusWaitTimeout);
         return false;
