@@ -115,7 +115,6 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
   constexpr uint32_t kTmemCols = 512;
   constexpr uint32_t kColS = 0, kColdP = 128, kColdS = 256, kColQ = 320, kColdQ = 384;
   constexpr int kMmaWarp = 4 * kDqGroups, kTmaWarp = 4 * kDqGroups + 1;
-  constexpr int kHalfBytes = 64 * 128;  // 64 rows of a block
   const int n_tiles = seg_tiles(segs);
 
   if (tid == 0) {
