@@ -26,13 +26,13 @@ constexpr int kFwdThreads = 128 * kFwdGroups + 64;
 template <int D> struct FwdSmem {
   static constexpr int kK = 0;
   static constexpr int kV = kK + kFwdKStages * TileGeom<D>::kBytes;
-  static constexpr int kMax = kV + kFwdVStages * TileGeom<D>::kBytes;  // float [2 tile parities][groups][128]
-  static constexpr int kBars = kMax + 2 * kFwdGroups * kTile * 4;
+  static constexpr int kMax = kV + kFwdVStages * TileGeom<D>::kBytes;  // float [2 parities + 1][groups][128]
+  static constexpr int kBars = kMax + 3 * kFwdGroups * kTile * 4;
   static constexpr int kTotal = kBars + 256 + 1024;  // barriers, tmem holder, abort flag + slack to align to 1024
 };
 
 constexpr int kPolyOf8 = 2;  // of every 8 pairs of exponentials, how many use the polynomial on the FMA pipe
-constexpr float kRescaleThreshold = 8.0f;  // log2 units: stale row max tolerated before O is rescaled
+constexpr float kRowSumLimit = 1073741824.f;  // 2^30: a tile row sum beyond it makes the row re-reference itself
 
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
@@ -201,112 +201,121 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
       mbar_wait(s_full + buf, (j / kFwdSBufs) & 1, abort_flag);
       tc_fence_after_sync();
 
-      uint32_t s[NL][32];
+      // P = exp2(s * scale * log2e - m_run) for this thread's keys, with the row sum; m_run is whatever
+      // reference the row has had so far (any reference is exact as long as nothing overflows)
+      auto exponentiate = [&](uint32_t (&pk)[NL][16]) -> float {
+        uint32_t s[NL][32];
 #pragma unroll
-      for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);
-      tmem_wait_ld();
-      float mx;
-      if (valid < kFwdCols) {
-        mx = -INFINITY;
+        for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);
+        tmem_wait_ld();
+        const float neg_m = -m_run;
+        float rowsum;
+        if (valid < kFwdCols) {
+          rowsum = 0.f;
+#pragma unroll
+          for (int c2 = 0; c2 < NL; ++c2)
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+              float p0 = fast_exp2(fmaf(__uint_as_float(s[c2][c]), scale_log2, neg_m));
+              float p1 = fast_exp2(fmaf(__uint_as_float(s[c2][c + 1]), scale_log2, neg_m));
+              if (c2 * 32 + c >= valid) p0 = 0.f;
+              if (c2 * 32 + c + 1 >= valid) p1 = 0.f;
+              rowsum += p0 + p1;
+              pk[c2][c >> 1] = pack_bf16(p0, p1);
+            }
+        } else {
+          // full tile: packed fp32 arithmetic; kPolyOf8 of every 8 pairs take the polynomial exp2
+          const uint64_t sc2 = f32x2(scale_log2, scale_log2), nm2 = f32x2(neg_m, neg_m);
+          uint64_t acc_a = f32x2(0.f, 0.f), acc_b = f32x2(0.f, 0.f);
+#pragma unroll
+          for (int c2 = 0; c2 < NL; ++c2)
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+              const uint64_t x2 = fma2(f32x2(__uint_as_float(s[c2][c]), __uint_as_float(s[c2][c + 1])), sc2, nm2);
+              float p0, p1;
+              if (((c >> 1) & 7) < kPolyOf8) {
+                exp2_poly_pair(x2, p0, p1);
+              } else {
+                float x0, x1;
+                f32x2_split(x2, x0, x1);
+                p0 = fast_exp2(x0);
+                p1 = fast_exp2(x1);
+              }
+              if ((c >> 1) & 1) acc_a = add2(acc_a, f32x2(p0, p1));
+              else acc_b = add2(acc_b, f32x2(p0, p1));
+              pk[c2][c >> 1] = pack_bf16(p0, p1);
+            }
+          float r0, r1;
+          f32x2_split(add2(acc_a, acc_b), r0, r1);
+          rowsum = r0 + r1;
+        }
+        return rowsum;
+      };
+
+      // Fast path: no row maximum at all.  The tile is exponentiated against the row's current reference;
+      // only if a row sum leaves the safe range (or the row has no reference yet: first tile) does the row take
+      // the true maximum of the tile as its new reference.  The two threads of a row must agree, so each
+      // publishes its verdict and reads the other's (one 64-thread barrier per warp pair and tile).
+      uint32_t pk[NL][16];
+      float rowsum = 0.f;
+      bool redo = m_run == -INFINITY;
+      if (!__all_sync(0xffffffffu, redo)) {
+        rowsum = exponentiate(pk);
+        redo = redo || !(rowsum < kRowSumLimit);   // also true for inf and NaN
+      }
+      float* fslot = smax + (j & 1) * kFwdGroups * kTile;
+      fslot[g * kTile + r] = redo ? 1.f : 0.f;
+      named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
+#pragma unroll
+      for (int og = 0; og < kFwdGroups; ++og) redo = redo || fslot[og * kTile + r] != 0.f;
+      float alpha = 1.f;
+      if (__any_sync(0xffffffffu, redo)) {
+        // Slow path (first tile, or scores far above everything seen so far): exact tile maximum, shared
+        // between the threads of the row; rows of the warp that did not ask for it keep their reference.
+        uint32_t s[NL][32];
+#pragma unroll
+        for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);   // S is still intact
+        tmem_wait_ld();
+        float mx = -INFINITY;
 #pragma unroll
         for (int c2 = 0; c2 < NL; ++c2)
 #pragma unroll
           for (int c = 0; c < 32; ++c)
             if (c2 * 32 + c < valid) mx = fmaxf(mx, __uint_as_float(s[c2][c]));
-      } else {
-        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+        float* mslot = smax + 2 * kFwdGroups * kTile;
+        mslot[g * kTile + r] = mx;
+        named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
 #pragma unroll
-        for (int c2 = 0; c2 < NL; ++c2)
+        for (int og = 0; og < kFwdGroups; ++og) mx = fmaxf(mx, mslot[og * kTile + r]);  // finite: >= 1 valid key
+        if (redo) {
+          const float m_new = mx * scale_log2;
+          if (m_run != -INFINITY) alpha = fast_exp2(m_run - m_new);   // may be > 1 if the max went down: exact too
+          m_run = m_new;
+        }
+        if (j > 0) {
+          // O must be at rest: wait for the P V of the previous tile.  The barriers alternate with the tile
+          // parity, so the awaited phase is at most one completion away.
+          mbar_wait(pv_done + ((j - 1) & 1), ((j - 1) >> 1) & 1, abort_flag);
+          tc_fence_after_sync();
+          // 32-column slices of the row are dealt round-robin to the groups
 #pragma unroll
-          for (int c = 0; c < 32; c += 8) {
-            mx0 = max3(mx0, __uint_as_float(s[c2][c]), __uint_as_float(s[c2][c + 1]));
-            mx1 = max3(mx1, __uint_as_float(s[c2][c + 2]), __uint_as_float(s[c2][c + 3]));
-            mx2 = max3(mx2, __uint_as_float(s[c2][c + 4]), __uint_as_float(s[c2][c + 5]));
-            mx3 = max3(mx3, __uint_as_float(s[c2][c + 6]), __uint_as_float(s[c2][c + 7]));
+          for (int c4 = 0; c4 < D / 32; ++c4) {
+            if (c4 % kFwdGroups != g) continue;
+            uint32_t acc[32];
+            tmem_ld32(tmem_lane + kColO + c4 * 32, acc);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) acc[c] = __float_as_uint(__uint_as_float(acc[c]) * alpha);
+            tmem_st32(tmem_lane + kColO + c4 * 32, acc);
           }
-        mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        }
+        l_run *= alpha;
+        rowsum = exponentiate(pk);
       }
-      // the thread of the other group that owns the same row contributes the max of its half of the tile;
-      // both then take identical decisions about the running max (warps w and w+4 hold the same rows)
-      float* mslot = smax + (j & 1) * kFwdGroups * kTile;
-      mslot[g * kTile + r] = mx;
-      named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
-#pragma unroll
-      for (int og = 0; og < kFwdGroups; ++og) mx = fmaxf(mx, mslot[og * kTile + r]);  // finite: >= 1 valid key
-      const float m_new = mx * scale_log2;
-      float alpha = 1.f;
-      bool rescale = false;
-      if (m_run == -INFINITY) {
-        m_run = m_new;                        // first tile: O holds nothing yet
-      } else if (m_new - m_run > kRescaleThreshold) {
-        alpha = fast_exp2(m_run - m_new);
-        m_run = m_new;
-        rescale = true;
-      }
-      const float neg_m = -m_run;
-      float rowsum;
-      uint32_t pk[NL][16];
-      if (valid < kFwdCols) {
-        rowsum = 0.f;
-#pragma unroll
-        for (int c2 = 0; c2 < NL; ++c2)
-#pragma unroll
-          for (int c = 0; c < 32; c += 2) {
-            float p0 = fast_exp2(fmaf(__uint_as_float(s[c2][c]), scale_log2, neg_m));
-            float p1 = fast_exp2(fmaf(__uint_as_float(s[c2][c + 1]), scale_log2, neg_m));
-            if (c2 * 32 + c >= valid) p0 = 0.f;
-            if (c2 * 32 + c + 1 >= valid) p1 = 0.f;
-            rowsum += p0 + p1;
-            pk[c2][c >> 1] = pack_bf16(p0, p1);
-          }
-      } else {
-        // full tile: packed fp32 arithmetic; kPolyOf8 of every 8 pairs take the polynomial exp2 so that the
-        // special-function unit and the FMA pipe share the exponentials
-        const uint64_t sc2 = f32x2(scale_log2, scale_log2), nm2 = f32x2(neg_m, neg_m);
-        uint64_t acc_a = f32x2(0.f, 0.f), acc_b = f32x2(0.f, 0.f);
-#pragma unroll
-        for (int c2 = 0; c2 < NL; ++c2)
-#pragma unroll
-          for (int c = 0; c < 32; c += 2) {
-            const uint64_t x2 = fma2(f32x2(__uint_as_float(s[c2][c]), __uint_as_float(s[c2][c + 1])), sc2, nm2);
-            float p0, p1;
-            if (((c >> 1) & 7) < kPolyOf8) {
-              exp2_poly_pair(x2, p0, p1);
-            } else {
-              float x0, x1;
-              f32x2_split(x2, x0, x1);
-              p0 = fast_exp2(x0);
-              p1 = fast_exp2(x1);
-            }
-            if ((c >> 1) & 1) acc_a = add2(acc_a, f32x2(p0, p1));
-            else acc_b = add2(acc_b, f32x2(p0, p1));
-            pk[c2][c >> 1] = pack_bf16(p0, p1);
-          }
-        float r0, r1;
-        f32x2_split(add2(acc_a, acc_b), r0, r1);
-        rowsum = r0 + r1;
-      }
-      l_run = l_run * alpha + rowsum;
+      l_run += rowsum;
 #pragma unroll
       for (int c2 = 0; c2 < NL; ++c2)   // in place: this thread has read all of its S columns
         tmem_st16(tmem_lane + colS + c2 * 16, pk[c2]);
-      if (__any_sync(0xffffffffu, rescale)) {
-        // O must be at rest: wait for the PV of the previous tile (rescale implies j >= 1).  The barriers
-        // alternate with the tile parity, so the awaited phase is at most one completion away.
-        mbar_wait(pv_done + ((j - 1) & 1), ((j - 1) >> 1) & 1, abort_flag);
-        tc_fence_after_sync();
-        // 32-column slices of the row are dealt round-robin to the groups
-#pragma unroll
-        for (int c4 = 0; c4 < D / 32; ++c4) {
-          if (c4 % kFwdGroups != g) continue;
-          uint32_t acc[32];
-          tmem_ld32(tmem_lane + kColO + c4 * 32, acc);
-          tmem_wait_ld();
-#pragma unroll
-          for (int c = 0; c < 32; ++c) acc[c] = __float_as_uint(__uint_as_float(acc[c]) * alpha);
-          tmem_st32(tmem_lane + kColO + c4 * 32, acc);
-        }
-      }
       if (g == 0 && tile_valid < kTile) {
         // Rows past the segment's end may hold stale cache contents: P is 0 there, but 0 * NaN is NaN.
         // Group 0 clears them before publishing P_0, which both PV MMAs of the tile are issued after.
