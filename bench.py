@@ -70,7 +70,7 @@ def aggregate(flops_per_rank_step: float, ms_per_step_max: float, world: int) ->
 class ClockSampler:
     """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw,power.limit")
     NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
 
     def __init__(self, gpu_id: str):
@@ -101,7 +101,7 @@ class ClockSampler:
             self.proc.wait(timeout=2)
         except Exception:
             self.proc.kill()
-        mhz, mx, reasons = [], None, set()
+        mhz, mx, reasons, watts, limit = [], None, set(), [], None
         for ts, line in self.lines:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 6 or not (t0 <= ts <= t1 + 0.05):
@@ -110,6 +110,10 @@ class ClockSampler:
                 mhz.append(float(parts[0])); mx = float(parts[1])
             except ValueError:
                 continue
+            try:
+                watts.append(float(parts[6])); limit = float(parts[7])
+            except (ValueError, IndexError):
+                pass
             for name, val in zip(self.NAMES, parts[2:6]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
@@ -121,7 +125,7 @@ class ClockSampler:
                 except (ValueError, IndexError):
                     pass
         return {"sm_mhz": float(np.median(mhz)) if mhz else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(mhz)}
+                "samples": len(mhz), "power_w": float(np.median(watts)) if watts else None, "power_limit_w": limit}
 
 
 # ----------------------------------------------------------------------------------------------- CPU oracle leg

@@ -316,3 +316,29 @@ def test_random_shapes_and_cache_histories(seed):
     loose = scale > 0.2          # sharper softmax: outputs of magnitude ~|v| (see the scale 0.7 case above)
     _run_case(A, B, Bc, H, D, T, S, L, held, n_q, n_kc, 20000 + 100 * seed, churn=churn, evict_hole=hole, scale=scale,
               o_max_abs=1.8e-2 if loose else 1e-2, o_mean_abs=2.5e-3 if loose else 1e-3)
+
+
+@pytest.mark.parametrize("order", ["rising", "falling", "spike"])
+def test_row_reference_follows_score_jumps_between_tiles(order):
+    """The forward takes no row maximum on its fast path: a row re-references itself only when a tile's row sum
+    leaves the safe range.  Here later key tiles score far above (or below) earlier ones, so that path runs
+    several times per row (rising), never after the first tile (falling), or once in the middle (spike)."""
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, n_q, n_k = 1, 2, 128, 200, 128 * 6 + 40
+    qb = synth.normal_bf16(4101, (B, n_q, H, D)); kb = synth.normal_bf16(4102, (B, n_k, H, D))
+    vb = synth.normal_bf16(4103, (B, n_k, H, D)); dob = synth.normal_bf16(4104, (B, n_q, H, D))
+    kf = orc.bf16_bits_to_f64(kb)
+    tile = np.arange(n_k) // 128
+    gain = {"rising": 1.0 + 1.5 * tile, "falling": 10.0 - 1.5 * tile, "spike": np.where(tile == 3, 12.0, 1.0)}[order]
+    kb = synth.f32_to_bf16_bits((kf * gain[None, :, None, None]).astype(np.float32))   # exact in bf16? re-round
+    kf = orc.bf16_bits_to_f64(kb)
+    q, k, v, do = (dev_bf16(x) for x in (qb, kb, vb, dob))
+    qf, vf, dof = (orc.bf16_bits_to_f64(x) for x in (qb, vb, dob))
+    scale = 1.0 / np.sqrt(D)
+    o, lse = A.astro_chunk_attn_fwd(None, q, k, v, scale)
+    A.astro_last_device_status()
+    o_ref, lse_ref = orc.chunk_attn_fwd(qf, None, None, kf, vf, scale)
+    # near one-hot rows: the output is about one V row, tolerance as in the sharp-softmax case above
+    check_fwd(o, lse, o_ref, lse_ref, o_max_abs=1.8e-2, o_mean_abs=2.5e-3)
+    g = A.astro_chunk_attn_bwd(None, q, k, v, o, lse, do, scale)
+    check_grads(g, orc.chunk_attn_bwd(qf, None, None, kf, vf, dof, scale))
