@@ -6,10 +6,12 @@
 // Q lives in tensor memory (bf16 pairs, written once by the softmax threads) and is the A operand of
 // S = Q K^T, so shared memory only carries K and V: an MMA with both operands in shared memory reads
 // 128 B/clk, the whole shared-memory bandwidth, and then competes with the TMA writes of the next tiles.
-// S of a whole key tile is one 128x128 MMA into one of two S buffers, issued two tiles ahead.  The threads that share a query row (one per group)
-// exchange their tile maxima through shared memory and keep the same running max, so all parts of
-// P V accumulate into ONE O accumulator; each keeps its own partial row sum.  P is written as bf16 pairs
-// over the thread's own S columns.  K and V tiles travel through 3-deep rings.
+// S of a whole key tile is one 128x128 MMA into one of two S buffers, issued two tiles ahead.
+// The threads that share a query row (one per group) keep the same reference exponent for the row, so all
+// parts of P V accumulate into ONE O accumulator; each keeps its own partial row sum.  The fast path takes
+// no row maximum: a row re-references itself (true tile maximum, O and row sums rescaled) only when a tile's
+// row sum leaves the safe range.  P is written as bf16 pairs over the thread's own S columns.  K and V tiles
+// travel through 3-deep rings.
 // Part of the exponentials is evaluated by a polynomial on the FMA pipe, because the special-function
 // unit (16 exp2 per clock per SM) is as busy as the tensor core at head_dim 128.
 //   TMEM columns: S buffers [0,128) [128,256)   O [256,256+D)   Q [384,384+D/2)
