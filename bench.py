@@ -350,8 +350,8 @@ def run_ours(args):
     kname, kflops = kernel_flops[dom]
     achieved = kflops / (stage_ms[dom] * 1e-3) / 1e12
     peak = peaks["bf16_sustained"]
-    # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
-    # profiles/attention_kernels_layer_shape.md; set an entry to None when its kernel changes.
+    # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu capture of these
+    # kernels on this workload; set an entry to None when its kernel changes.
     ncu_traffic = {"fwd": 232.95e6, "dq": 246.85e6, "dkv": 62.0e6}
     roofline = {"bound": "tensor", "kernel": kname, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": ncu_traffic[dom], "traffic_unit": "bytes of DRAM traffic per launch",

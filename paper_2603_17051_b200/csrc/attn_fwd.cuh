@@ -257,7 +257,7 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
       // Fast path: no row maximum at all.  The tile is exponentiated against the row's current reference;
       // only if a row sum leaves the safe range (or the row has no reference yet: first tile) does the row take
       // the true maximum of the tile as its new reference.  The two threads of a row must agree, so each
-      // publishes its verdict and reads the other's (one 64-thread barrier per warp pair and tile).
+      // publishes its decision and reads the other's (one 64-thread barrier per warp pair and tile).
       uint32_t pk[NL][16];
       float rowsum = 0.f;
       bool redo = m_run == -INFINITY;
