@@ -471,6 +471,29 @@ def run_extra(args):
                           "config": "B=4 H=12 D=128 T=1560, S=3 + %d window slots, 80 chunks x (evict, 4 fwd, append)" % slots,
                           "frac_of_bf16_sustained": flops / (ms * 1e-3) / 1e12 / peaks["bf16_sustained"]}))
         return 0
+    if args.workload == "variants":
+        # window presets of Tab. S1 (S = 3; L = 21 or 15 frames attended in total, the chunk included) with
+        # 3-frame chunks and with per-frame chunks: forward of one layer, batch 4
+        Bv = 4
+        for total, cf in ((21, 3), (21, 1), (15, 3), (15, 1)):
+            held, Mv = total - cf, cf * T
+            cache = A.astro_kvcache_create(Bv, H, D, T, 3, total - 3, device=dev)
+            A.astro_kvcache_append(cache, rnd(40, (Bv, held * T, H, D)), rnd(41, (Bv, held * T, H, D)), held)
+            qv, kv, vv = (rnd(42 + i, (Bv, Mv, H, D)) for i in range(3))
+            ov = torch.empty_like(qv); lv = torch.empty((Bv, H, Mv), dtype=torch.float32, device=dev)
+            sc = 1.0 / float(np.sqrt(D))
+            fwd = lambda: A.astro_chunk_attn_fwd(cache, qv, kv, vv, sc, o=ov, lse=lv)
+            for _ in range(3):
+                fwd()
+            ms = _event_ms(fwd, 20)
+            A.astro_last_device_status()
+            flops = 4.0 * Bv * H * Mv * (held * T + Mv) * D
+            print(json.dumps({"workload": "variants", "attended_frames": total, "chunk_frames": cf, "batch": Bv,
+                              "queries": Mv, "keys": held * T + Mv, "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                              "latent_frames_per_s_4_steps": Bv * cf / (4 * ms * 1e-3),
+                              "frac_of_bf16_sustained": flops / (ms * 1e-3) / 1e12 / peaks["bf16_sustained"]}))
+            del cache
+        return 0
     if args.workload == "nft":
         # policy loss + selective KL + gradient on the velocity tensors of a 3-frame window (16 x 60 x 104 latents)
         Bn, E = 96, 3 * 16 * 60 * 104
@@ -592,7 +615,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", choices=("layer", "rollout", "rl_update", "sweep", "group", "nft"), default="layer",
+    ap.add_argument("--workload", choices=("layer", "rollout", "rl_update", "sweep", "group", "nft", "variants"), default="layer",
                     help="layer (default): the contract line; the others print one JSON line per extra workload")
     ap.add_argument("--group", type=int, default=24, help="group workload: candidates G decoding against one prefix")
     ap.add_argument("--replicated", action="store_true",
