@@ -137,3 +137,22 @@ def test_state_record_round_trip_and_validation():
         assert L.astro_kvcache_set_state(h, C.byref(bad)) == 2
     assert L.astro_kvcache_set_state(h, None) == 1
     L.astro_kvcache_destroy(h)
+
+
+def test_header_compiles_as_c_and_links(tmp_path):
+    """include/astro.h is a C header: build a C99 program against it and the shared library, run it."""
+    import shutil
+    import subprocess
+    from paper_2603_17051_b200 import build as B
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    A.lib()
+    exe = str(tmp_path / "c_abi_check")
+    cmd = [gcc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(ROOT, "include"),
+           os.path.join(ROOT, "tests", "c_abi_check.c"), "-o", exe, "-L", B.LIB_DIR, "-lastro",
+           "-Wl,-rpath," + B.LIB_DIR]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
+    run = subprocess.run([exe], capture_output=True, text=True)
+    assert run.returncode == 0 and "c abi ok" in run.stdout, run.stdout + run.stderr
