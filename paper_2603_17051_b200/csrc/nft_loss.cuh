@@ -9,7 +9,7 @@
 namespace astro {
 
 constexpr int kNftThreads = 256;
-constexpr int kNftVecsPerThread = 4;  // 4 x 8 bf16 per tensor in flight per thread
+constexpr int kNftVecsPerThread = 1;  // measured: one 16-byte vector per tensor and thread (many small blocks) is fastest
 
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&f)[8]) {
   const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
