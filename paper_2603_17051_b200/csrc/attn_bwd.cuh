@@ -446,14 +446,18 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const float scale_log2 = scale * kLog2e;
     const uint64_t sc2 = f32x2(scale_log2, scale_log2);
     const size_t stat_base = (static_cast<size_t>(b) * heads + h) * n_q;
+    // per-query constants (LSE * log2e, delta) of this group's 64 queries, fetched one tile ahead so that the
+    // global-memory latency is off the critical path; +inf as LSE turns rows past n_q into P = 0
+    auto fetch_stat = [&](int i) -> float2 {
+      const int qi = i * kTile + g * 64 + r;
+      return (r < 64 && qi < n_q) ? make_float2(lse[stat_base + qi] * kLog2e, delta[stat_base + qi])
+                                  : make_float2(INFINITY, 0.f);
+    };
+    float2 stat_next = fetch_stat(0);
     for (int i = 0; i < n_tiles; ++i) {
-      // per-query constants of this group's 64 queries; +inf as LSE turns rows past n_q into P = 0
       float2* stat = sStat + (i & 1) * kTile + g * 64;
-      if (r < 64) {
-        const int qi = i * kTile + g * 64 + r;
-        stat[r] = qi < n_q ? make_float2(lse[stat_base + qi] * kLog2e, delta[stat_base + qi])
-                           : make_float2(INFINITY, 0.f);
-      }
+      if (r < 64) stat[r] = stat_next;
+      if (i + 1 < n_tiles) stat_next = fetch_stat(i + 1);
       named_barrier_sync(1 + g, 128);
       mbar_wait(s_full, i & 1, abort_flag);
       tc_fence_after_sync();
