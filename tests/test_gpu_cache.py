@@ -110,3 +110,24 @@ def test_saved_storage_and_state_resume_on_a_new_handle():
     A.astro_kvcache_append(resumed, dev_bf16(kb), dev_bf16(vb), 1); model.append(kb, vb, T)
     _both_export_equal(A, resumed, model)
     assert A.astro_kvcache_query(resumed)[2] == model.frames_seen
+
+
+def test_cache_storage_canaries_are_untouched():
+    """Appends at every ring position write inside the bound storage only (padding on both sides stays intact)."""
+    import torch
+    from paper_2603_17051_b200 import binding as A
+    Bc, H, D, T, S, L = 2, 3, 128, 11, 2, 3
+    nbytes = A.astro_kvcache_storage_bytes(Bc, H, D, T, S, L)
+    pad = 4096
+    bufs = [torch.full((nbytes + 2 * pad,), 0x5A, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    cache = A.astro_kvcache_create(Bc, H, D, T, S, L, k_storage=bufs[0][pad:pad + nbytes],
+                                   v_storage=bufs[1][pad:pad + nbytes])
+    model = orc.RollingKVCache(S, L)
+    for n in range(12):
+        if model.held() == S + L:
+            A.astro_kvcache_evict(cache, 1); model.evict(1)
+        kb = synth.normal_bf16(9300 + 2 * n, (Bc, T, H, D)); vb = synth.normal_bf16(9301 + 2 * n, (Bc, T, H, D))
+        A.astro_kvcache_append(cache, dev_bf16(kb), dev_bf16(vb), 1); model.append(kb, vb, T)
+    _both_export_equal(A, cache, model)
+    for b in bufs:
+        assert (b[:pad] == 0x5A).all() and (b[-pad:] == 0x5A).all()
