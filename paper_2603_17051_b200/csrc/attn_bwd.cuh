@@ -66,7 +66,7 @@ constexpr int kDqGroups = 2;                      // softmax groups: more warps 
 constexpr int kDqCols = kTile / kDqGroups;         // exp2 latency behind the arithmetic of the other warps
 constexpr int kDqSoftmaxThreads = 128 * kDqGroups;
 constexpr int kDqThreads = kDqSoftmaxThreads + 64;
-constexpr int kDqPolyOf8 = 2;  // share of the exponentials evaluated on the FMA pipe
+constexpr int kDqPolyOf8 = 0;  // share of the exponentials on the FMA pipe: none pays here under the power limit
 
 template <int D> struct DqSmem {
   static constexpr int kdO = 0;
