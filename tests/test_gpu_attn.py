@@ -342,3 +342,33 @@ def test_row_reference_follows_score_jumps_between_tiles(order):
     check_fwd(o, lse, o_ref, lse_ref, o_max_abs=1.8e-2, o_mean_abs=2.5e-3)
     g = A.astro_chunk_attn_bwd(None, q, k, v, o, lse, do, scale)
     check_grads(g, orc.chunk_attn_bwd(qf, None, None, kf, vf, dof, scale))
+
+
+def test_calls_follow_the_callers_stream():
+    """Work is enqueued on the stream that is current in torch: results on a side stream match the default one."""
+    import torch
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, T = 2, 2, 128, 40
+    cache = A.astro_kvcache_create(B, H, D, T, 1, 3)
+    side = torch.cuda.Stream()
+    k0, v0 = (dev_bf16(synth.normal_bf16(5100 + i, (B, 3 * T, H, D))) for i in range(2))
+    q, kc, vc, do = (dev_bf16(synth.normal_bf16(5110 + i, (B, 150, H, D))) for i in range(4))
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        A.astro_kvcache_append(cache, k0, v0, 3)
+        o1, l1 = A.astro_chunk_attn_fwd(cache, q, kc, vc, 0.09)
+        g1 = A.astro_chunk_attn_bwd(cache, q, kc, vc, o1, l1, do, 0.09)
+    side.synchronize()
+    o2, l2 = A.astro_chunk_attn_fwd(cache, q, kc, vc, 0.09)
+    g2 = A.astro_chunk_attn_bwd(cache, q, kc, vc, o2, l2, do, 0.09)
+    torch.cuda.synchronize()
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+    for a, b in zip(g1, g2):
+        assert torch.equal(a, b)
+
+
+def test_many_samples_one_head():
+    """Grid dimensions: a batch of 70 samples with a single head, shared and per-sample caches."""
+    from paper_2603_17051_b200 import binding as A
+    for Bc in (70, 1):
+        _run_case(A, B=70, Bc=Bc, H=1, D=64, T=8, S=1, L=2, held=3, n_q=20, n_kc=9, seed=5200 + Bc)
