@@ -372,3 +372,24 @@ def test_many_samples_one_head():
     from paper_2603_17051_b200 import binding as A
     for Bc in (70, 1):
         _run_case(A, B=70, Bc=Bc, H=1, D=64, T=8, S=1, L=2, held=3, n_q=20, n_kc=9, seed=5200 + Bc)
+
+
+def test_zero_scale_gives_uniform_attention():
+    """scale = 0: every key gets the same weight, O is the mean of all values, LSE = ln(number of keys)."""
+    import torch
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, T = 1, 2, 128, 50
+    cache = A.astro_kvcache_create(B, H, D, T, 0, 4)
+    kx, vx = (dev_bf16(synth.normal_bf16(5300 + i, (B, 4 * T, H, D))) for i in range(2))
+    A.astro_kvcache_append(cache, kx, vx, 4)
+    q, kc, vc, do = (dev_bf16(synth.normal_bf16(5310 + i, (B, 140, H, D))) for i in range(4))
+    o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, 0.0)
+    A.astro_last_device_status()
+    mean_v = torch.cat([vx, vc], dim=1).float().mean(dim=1, keepdim=True)
+    assert (o.float() - mean_v).abs().max() < 1e-2
+    assert (lse - float(np.log(4 * T + 140))).abs().max() < 1e-3
+    dq, dk, dv = A.astro_chunk_attn_bwd(cache, q, kc, vc, o, lse, do, 0.0)
+    A.astro_last_device_status()
+    assert dq.float().abs().max() == 0 and dk.float().abs().max() == 0          # both carry the factor scale
+    expect_dv = do.float().sum(dim=1, keepdim=True) / (4 * T + 140)
+    assert (dv.float() - expect_dv).abs().max() < 2e-2
