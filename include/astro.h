@@ -104,6 +104,14 @@ typedef struct {
 astro_status_t astro_kvcache_get_state(const astro_kvcache_t* cache, astro_kvcache_state_t* state);
 astro_status_t astro_kvcache_set_state(astro_kvcache_t* cache, const astro_kvcache_state_t* state);
 
+/* Inspection aid (host only, launches nothing): the physical token ranges of the cache storage that an
+ * attention call would walk in the cache's present state -- at most two, merged where adjacent, because the
+ * window ring can be split by its wrap-around or by a hole left by evict -- followed by the chunk's own keys
+ * when n_kc > 0.  HOST arrays of at least 3 entries each: first token, token count, and 1 for the chunk
+ * segment / 0 for a cache segment.  *n_segments receives the number of entries written. */
+astro_status_t astro_kvcache_key_segments(const astro_kvcache_t* cache, int n_kc, int* n_segments, int* first_token,
+                                          int* token_count, int* from_chunk);
+
 /* Inspection aid: write the held frames in logical order (sink frames, then
  * window oldest to newest) to k_out, v_out: device bf16 [B_c, held*T, H, D]. */
 astro_status_t astro_kvcache_export(const astro_kvcache_t* cache, void* k_out, void* v_out, void* stream);

@@ -16,7 +16,7 @@ STATUS_NAMES = {0: "ASTRO_OK", 1: "ASTRO_ERR_NULL", 2: "ASTRO_ERR_SHAPE", 3: "AS
                 4: "ASTRO_ERR_CAPACITY", 5: "ASTRO_ERR_UNDERFLOW", 6: "ASTRO_ERR_ARCH", 7: "ASTRO_ERR_CUDA",
                 8: "ASTRO_ERR_TIMEOUT"}
 
-EXPORTED = ("astro_selftest_wait_timeout", "astro_nft_loss", "astro_kvcache_get_state", "astro_kvcache_set_state", "astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcache_destroy", "astro_kvcache_reset",
+EXPORTED = ("astro_kvcache_key_segments", "astro_selftest_wait_timeout", "astro_nft_loss", "astro_kvcache_get_state", "astro_kvcache_set_state", "astro_kvcache_storage_bytes", "astro_kvcache_create", "astro_kvcache_destroy", "astro_kvcache_reset",
             "astro_kvcache_append", "astro_kvcache_evict", "astro_kvcache_query", "astro_kvcache_export",
             "astro_chunk_attn_fwd", "astro_chunk_attn_bwd_workspace_bytes", "astro_chunk_attn_bwd",
             "astro_chunk_attn_bwd_delta", "astro_chunk_attn_bwd_dq", "astro_chunk_attn_bwd_dkv",
@@ -70,6 +70,8 @@ def lib():
     L.astro_kvcache_get_state.argtypes = [vp, C.POINTER(KVCacheState)]
     L.astro_kvcache_set_state.restype = ci
     L.astro_kvcache_set_state.argtypes = [vp, C.POINTER(KVCacheState)]
+    L.astro_kvcache_key_segments.restype = ci
+    L.astro_kvcache_key_segments.argtypes = [vp, ci, C.POINTER(ci), C.POINTER(ci), C.POINTER(ci), C.POINTER(ci)]
     L.astro_kvcache_export.restype = ci
     L.astro_kvcache_export.argtypes = [vp, vp, vp, vp]
     L.astro_chunk_attn_fwd.restype = ci
@@ -198,6 +200,15 @@ def astro_kvcache_get_state(cache: KVCache) -> KVCacheState:
 
 def astro_kvcache_set_state(cache: KVCache, state: KVCacheState) -> None:
     _check(lib().astro_kvcache_set_state(cache.handle, C.byref(state)), "astro_kvcache_set_state")
+
+
+def astro_kvcache_key_segments(cache, n_kc: int):
+    """List of (first_token, token_count, from_chunk) the attention kernels would walk (host only)."""
+    n = C.c_int()
+    a, b, c = (C.c_int * 3)(), (C.c_int * 3)(), (C.c_int * 3)()
+    _check(lib().astro_kvcache_key_segments(None if cache is None else cache.handle, int(n_kc), C.byref(n), a, b, c),
+           "astro_kvcache_key_segments")
+    return [(a[i], b[i], c[i]) for i in range(n.value)]
 
 
 def astro_kvcache_export(cache: KVCache, stream=None):

@@ -377,6 +377,21 @@ astro_status_t astro_kvcache_set_state(astro_kvcache_t* c, const astro_kvcache_s
   return ASTRO_OK;
 }
 
+astro_status_t astro_kvcache_key_segments(const astro_kvcache_t* c, int n_kc, int* n_segments, int* first_token,
+                                          int* token_count, int* from_chunk) {
+  if (!n_segments || !first_token || !token_count || !from_chunk) return ASTRO_ERR_NULL;
+  if (n_kc < 0) return ASTRO_ERR_SHAPE;
+  const bool have_ctx = c && (c->sink_held + c->win_held) > 0;
+  const KeySegs s = build_segments(have_ctx ? c : nullptr, n_kc);
+  *n_segments = s.n;
+  for (int i = 0; i < s.n; ++i) {
+    first_token[i] = s.start[i];
+    token_count[i] = s.count[i];
+    from_chunk[i] = s.from_chunk[i];
+  }
+  return ASTRO_OK;
+}
+
 astro_status_t astro_kvcache_export(const astro_kvcache_t* c, void* k_out, void* v_out, void* stream) {
   if (!c || !k_out || !v_out) return ASTRO_ERR_NULL;
   if (!aligned16(k_out) || !aligned16(v_out)) return ASTRO_ERR_ALIGN;

@@ -156,3 +156,35 @@ def test_header_compiles_as_c_and_links(tmp_path):
     assert res.returncode == 0, res.stderr
     run = subprocess.run([exe], capture_output=True, text=True)
     assert run.returncode == 0 and "c abi ok" in run.stdout, run.stdout + run.stderr
+
+
+def test_key_segments_cover_exactly_the_held_slots_in_every_ring_state():
+    """Host logic the kernels rely on: for every (sink, ring head, window count) state the cache segments are
+    disjoint, at most two, merged where adjacent, and cover exactly the tokens of the held slots."""
+    L = A.lib()
+    for S, Lw, T in ((0, 1, 3), (0, 4, 5), (2, 3, 7), (3, 5, 2)):
+        st, h = _raw_create(A.KVCacheDesc(1, 1, 64, T, S, Lw))
+        assert st == 0
+        n, a, b, c = C.c_int(), (C.c_int * 3)(), (C.c_int * 3)(), (C.c_int * 3)()
+        states = [(sink, 0, 0) for sink in range(S + 1)] + [(S, head, held) for head in range(Lw) for held in range(1, Lw + 1)]
+        for sink, head, held in states:
+            rec = A.KVCacheState(sink, head, held, sink + held + 10)
+            assert L.astro_kvcache_set_state(h, C.byref(rec)) == 0
+            for n_kc in (0, 9):
+                assert L.astro_kvcache_key_segments(h, n_kc, C.byref(n), a, b, c) == 0
+                segs = [(a[i], b[i], c[i]) for i in range(n.value)]
+                cache_segs = [s for s in segs if s[2] == 0]
+                chunk_segs = [s for s in segs if s[2] == 1]
+                assert chunk_segs == ([(0, n_kc, 1)] if n_kc else []) and (not chunk_segs or segs[-1] == chunk_segs[0])
+                assert len(cache_segs) <= 2
+                slots = list(range(sink)) + [S + (head + i) % Lw for i in range(held)]
+                expect = sorted(t for sl in slots for t in range(sl * T, (sl + 1) * T))
+                got = sorted(t for f, cnt, _ in cache_segs for t in range(f, f + cnt))
+                assert got == expect, (S, Lw, sink, head, held)
+                assert len(set(got)) == len(got)
+                cache_segs.sort()
+                for x, y in zip(cache_segs, cache_segs[1:]):
+                    assert x[0] + x[1] < y[0]                      # adjacent ranges were merged
+        L.astro_kvcache_destroy(h)
+    # no cache at all: only the chunk
+    assert A.astro_kvcache_key_segments(None, 5) == [(0, 5, 1)]
