@@ -371,7 +371,9 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
 
   if (tid == 0) {
     mbar_init(kv_full, 1);
-    for (int i = 0; i < kDkvStages; ++i) { mbar_init(q_full + i, 1); mbar_init(q_empty + i, 1); }
+    // a (Q, dO) stage is full when its TMA bytes have landed and the producer warp has staged the per-query
+    // constants of the tile beside it: two arrivals
+    for (int i = 0; i < kDkvStages; ++i) { mbar_init(q_full + i, 2); mbar_init(q_empty + i, 1); }
     mbar_init(s_full, 1);
     mbar_init(dp_full, 1);
     mbar_init(p_full, 256);
@@ -391,17 +393,31 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
   const uint32_t tmem_base = *tmem_holder;
 
   if (warp == kTmaWarp) {
+    // the whole warp: lane 0 issues the TMA loads, every lane stages the (LSE * log2e, delta) pairs of four
+    // queries of the tile; +inf as LSE turns query rows past n_q into P = 0
+    const size_t stat_base = (static_cast<size_t>(b) * heads + h) * n_q;
     if (lane == 0) {
       mbar_arrive_expect_tx(kv_full, 2 * TileGeom<D>::kBytes);
       tma_load_tile<D>(sK, &tm_kc, kv_full, k0, h, b);
       tma_load_tile<D>(sV, &tm_vc, kv_full, k0, h, b);
-      for (int i = 0; i < n_tiles; ++i) {
-        const int st = i % kDkvStages;
-        mbar_wait_spin(q_empty + st, ((i / kDkvStages) & 1) ^ 1, abort_flag);
+    }
+    for (int i = 0; i < n_tiles; ++i) {
+      const int st = i % kDkvStages;
+      mbar_wait(q_empty + st, ((i / kDkvStages) & 1) ^ 1, abort_flag);
+      if (lane == 0) {
         mbar_arrive_expect_tx(q_full + st, 2 * TileGeom<D>::kBytes);
         tma_load_tile<D>(sQ + st * TileGeom<D>::kBytes, &tm_q, q_full + st, i * kTile, h, b);
         tma_load_tile<D>(sdO + st * TileGeom<D>::kBytes, &tm_do, q_full + st, i * kTile, h, b);
       }
+      float2* stat = sStat + st * kTile;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int qi = i * kTile + lane * 4 + e;
+        stat[lane * 4 + e] = qi < n_q ? make_float2(lse[stat_base + qi] * kLog2e, delta[stat_base + qi])
+                                      : make_float2(INFINITY, 0.f);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(q_full + st);
     }
   } else if (warp == kMmaWarp) {
     if (lane == 0) {
@@ -445,20 +461,10 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const float scale_log2 = scale * kLog2e;
     const uint64_t sc2 = f32x2(scale_log2, scale_log2);
-    const size_t stat_base = (static_cast<size_t>(b) * heads + h) * n_q;
-    // per-query constants (LSE * log2e, delta) of this group's 64 queries, fetched one tile ahead so that the
-    // global-memory latency is off the critical path; +inf as LSE turns rows past n_q into P = 0
-    auto fetch_stat = [&](int i) -> float2 {
-      const int qi = i * kTile + g * 64 + r;
-      return (r < 64 && qi < n_q) ? make_float2(lse[stat_base + qi] * kLog2e, delta[stat_base + qi])
-                                  : make_float2(INFINITY, 0.f);
-    };
-    float2 stat_next = fetch_stat(0);
     for (int i = 0; i < n_tiles; ++i) {
-      float2* stat = sStat + (i & 1) * kTile + g * 64;
-      if (r < 64) stat[r] = stat_next;
-      if (i + 1 < n_tiles) stat_next = fetch_stat(i + 1);
-      named_barrier_sync(1 + g, 128);
+      // per-query constants of this group's 64 queries, staged by the producer warp with the tile
+      const float2* stat = sStat + (i % kDkvStages) * kTile + g * 64;
+      mbar_wait(q_full + i % kDkvStages, (i / kDkvStages) & 1, abort_flag);
       mbar_wait(s_full, i & 1, abort_flag);
       tc_fence_after_sync();
       uint32_t s[2][32], pt[32];
