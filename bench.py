@@ -352,7 +352,7 @@ def run_ours(args):
     peak = peaks["bf16_sustained"]
     # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu capture of these
     # kernels on this workload; set an entry to None when its kernel changes.
-    ncu_traffic = {"fwd": 231.13e6, "dq": 247.19e6, "dkv": 61.35e6}
+    ncu_traffic = {"fwd": 232.21e6, "dq": 247.52e6, "dkv": 61.34e6}
     roofline = {"bound": "tensor", "kernel": kname, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": ncu_traffic[dom], "traffic_unit": "bytes of DRAM traffic per launch",
                 "peak_source": "%s bf16 sustained (kernel timed inside a long loop); burst %.1f" % (peaks["source"], peaks["bf16_burst"]),
