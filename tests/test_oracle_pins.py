@@ -251,3 +251,21 @@ def test_cache_model_sink_retention_and_window_order():
         cache.append(frames[0], frames[0], T)
     with pytest.raises(IndexError):
         cache.evict(L + 1)
+
+
+def test_tiny_stream_matches_stored_oracle_values():
+    """Regression guard: the oracle's results on the tiny streamed workload equal the stored values written by
+    tests/golden/make_tiny_expected.py (which calls only the oracle)."""
+    import importlib.util
+    import os
+    here = os.path.dirname(os.path.abspath(__file__))
+    spec = importlib.util.spec_from_file_location("make_tiny_expected", os.path.join(here, "golden", "make_tiny_expected.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    got = mod.tiny_stream_summaries()
+    lines = [l.split() for l in open(os.path.join(here, "golden", "tiny_stream_expected.txt")) if not l.startswith("#")]
+    assert len(lines) == len(got) == 20
+    for (n, name, s, a, e7, e3), ln in zip(got, lines):
+        assert int(ln[0]) == n and ln[1] == name
+        for val, txt in zip((s, a, e7, e3), ln[2:]):
+            assert abs(val - float(txt)) <= 1e-10 * max(1.0, abs(val)), (n, name)
