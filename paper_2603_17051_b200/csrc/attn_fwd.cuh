@@ -179,16 +179,18 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
     const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
     const int row = q0 + r;
     const bool in_range = row < n_q;
-    // Q row -> tensor memory: group g writes elements [64g, 64g+64) of its row as 32 packed columns
-    if (g * 64 < D) {
+    // Q row -> tensor memory: 64-element halves of the row (32 packed columns each) are dealt to the groups
+#pragma unroll
+    for (int hq = 0; hq < D / 64; ++hq) {
+      if (hq % kFwdGroups != g) continue;
       uint32_t qr[32];
-      const uint4* src = reinterpret_cast<const uint4*>(q + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + g * 64);
+      const uint4* src = reinterpret_cast<const uint4*>(q + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + hq * 64);
 #pragma unroll
       for (int v = 0; v < 8; ++v) {
         const uint4 t = in_range ? src[v] : make_uint4(0, 0, 0, 0);
         qr[4 * v] = t.x; qr[4 * v + 1] = t.y; qr[4 * v + 2] = t.z; qr[4 * v + 3] = t.w;
       }
-      tmem_st32(tmem_lane + kColQ + g * 32, qr);
+      tmem_st32(tmem_lane + kColQ + hq * 32, qr);
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(q_full);
