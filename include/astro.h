@@ -125,8 +125,9 @@ astro_status_t astro_kvcache_export(const astro_kvcache_t* cache, void* k_out, v
  * q [batch, n_q, H, D], k_chunk/v_chunk [batch, n_kc, H, D] (may be null when
  * n_kc = 0), o [batch, n_q, H, D] bf16, lse [batch, H, n_q] fp32 (may be null).
  * cache may be null (no context).  n_q, n_kc are token counts and need not be
- * multiples of T or of any tile.  ASTRO_ERR_SHAPE if there is no key at all, or
- * batch differs from B_c and B_c != 1.  bf16 products, fp32 accumulation and softmax. */
+ * multiples of T or of any tile.  ASTRO_ERR_SHAPE if there is no key at all,
+ * batch differs from B_c and B_c != 1, or scale is negative or not finite.
+ * bf16 products, fp32 accumulation and softmax. */
 astro_status_t astro_chunk_attn_fwd(const astro_kvcache_t* cache, const void* q, const void* k_chunk,
                                     const void* v_chunk, int batch, int heads, int head_dim, int n_q,
                                     int n_kc, float scale, void* o, float* lse, void* stream);
