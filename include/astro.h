@@ -217,6 +217,14 @@ astro_status_t astro_last_device_status(uint32_t* detail);
  * context stays usable.  Nothing faults or hangs. */
 astro_status_t astro_selftest_wait_timeout(void* stream);
 
+/* Diagnostic switch (the paper has no counterpart).  The forward kernel first runs a fast pass in which a
+ * query row keeps the maximum of its first key tile as its one reference exponent, and repeats a 128-query
+ * tile with a running reference (the "safe pass") only if a row sum left the range fp32 can hold.  enable != 0
+ * makes every later astro_chunk_attn_fwd of this process run the safe pass only; 0 restores normal operation.
+ * Results agree within the rounding of bf16 either way; the switch exists so that tests can cover the safe
+ * pass on ordinary inputs.  Process-wide, not stream-ordered: it applies to calls made after it returns. */
+astro_status_t astro_debug_forward_safe_only(int enable);
+
 /* Static, never null. */
 const char* astro_status_string(astro_status_t status);
 

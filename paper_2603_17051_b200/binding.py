@@ -20,7 +20,7 @@ EXPORTED = ("astro_kvcache_key_segments", "astro_selftest_wait_timeout", "astro_
             "astro_kvcache_append", "astro_kvcache_evict", "astro_kvcache_query", "astro_kvcache_export",
             "astro_chunk_attn_fwd", "astro_chunk_attn_bwd_workspace_bytes", "astro_chunk_attn_bwd",
             "astro_chunk_attn_bwd_delta", "astro_chunk_attn_bwd_dq", "astro_chunk_attn_bwd_dkv",
-            "astro_chunk_attn_bwd_static",
+            "astro_chunk_attn_bwd_static", "astro_debug_forward_safe_only",
             "astro_last_device_status", "astro_status_string")
 
 
@@ -90,6 +90,8 @@ def lib():
     L.astro_chunk_attn_bwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
     L.astro_nft_loss.restype = ci
     L.astro_nft_loss.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, C.c_longlong, cf, vp, vp, vp, vp]
+    L.astro_debug_forward_safe_only.restype = ci
+    L.astro_debug_forward_safe_only.argtypes = [ci]
     L.astro_selftest_wait_timeout.restype = ci
     L.astro_selftest_wait_timeout.argtypes = [vp]
     L.astro_last_device_status.restype = ci
@@ -117,6 +119,22 @@ def _stream(stream):
     import torch
     s = torch.cuda.current_stream() if stream is None else stream
     return C.c_void_p(s.cuda_stream)
+
+
+def _contiguous(*tensors):
+    for t in tensors:
+        if t is not None and not t.is_contiguous():
+            raise ValueError("tensor arguments must be contiguous")
+
+
+def _used_on(stream, *tensors):
+    """Tensors this wrapper allocated are used by kernels on `stream`: tell torch's caching allocator, so that
+    a block dropped by the caller is not handed out again (on the allocating stream) while they still run."""
+    if stream is None:
+        return
+    for t in tensors:
+        if t is not None:
+            t.record_stream(stream)
 
 
 def _desc(cache_batch, heads, head_dim, tokens_per_frame, sink_frames, window_frames):
@@ -229,12 +247,13 @@ def astro_chunk_attn_fwd(cache, q, k_chunk, v_chunk, scale: float, o=None, lse=N
     import torch
     B, n_q, H, D = q.shape
     n_kc = 0 if k_chunk is None else k_chunk.shape[1]
+    fresh = []
     if o is None:
-        o = torch.empty_like(q)
+        o = torch.empty_like(q); fresh.append(o)
     if lse is None:
-        lse = torch.empty((B, H, n_q), dtype=torch.float32, device=q.device)
-    for t in (q, k_chunk, v_chunk, o, lse):
-        assert t is None or t.is_contiguous()
+        lse = torch.empty((B, H, n_q), dtype=torch.float32, device=q.device); fresh.append(lse)
+    _contiguous(q, k_chunk, v_chunk, o, lse)
+    _used_on(stream, *fresh)
     st = lib().astro_chunk_attn_fwd(None if cache is None else cache.handle, _ptr(q), _ptr(k_chunk), _ptr(v_chunk),
                                     B, H, D, n_q, n_kc, float(scale), _ptr(o), _ptr(lse), _stream(stream))
     _check(st, "astro_chunk_attn_fwd")
@@ -251,17 +270,18 @@ def astro_chunk_attn_bwd(cache, q, k_chunk, v_chunk, o, lse, d_o, scale: float, 
     import torch
     B, n_q, H, D = q.shape
     n_kc = 0 if k_chunk is None else k_chunk.shape[1]
+    fresh = []
     if dq is None:
-        dq = torch.empty_like(q)
+        dq = torch.empty_like(q); fresh.append(dq)
     if n_kc and dk_chunk is None:
-        dk_chunk = torch.empty_like(k_chunk)
+        dk_chunk = torch.empty_like(k_chunk); fresh.append(dk_chunk)
     if n_kc and dv_chunk is None:
-        dv_chunk = torch.empty_like(v_chunk)
+        dv_chunk = torch.empty_like(v_chunk); fresh.append(dv_chunk)
     need = astro_chunk_attn_bwd_workspace_bytes(B, H, n_q, D)
     if workspace is None:
-        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
-    for t in (q, k_chunk, v_chunk, o, lse, d_o, dq, dk_chunk, dv_chunk):
-        assert t is None or t.is_contiguous()
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device); fresh.append(workspace)
+    _contiguous(q, k_chunk, v_chunk, o, lse, d_o, dq, dk_chunk, dv_chunk)
+    _used_on(stream, *fresh)
     st = lib().astro_chunk_attn_bwd(None if cache is None else cache.handle, _ptr(q), _ptr(k_chunk), _ptr(v_chunk),
                                     _ptr(o), _ptr(lse), _ptr(d_o), B, H, D, n_q, n_kc, float(scale), _ptr(dq),
                                     _ptr(dk_chunk), _ptr(dv_chunk), _ptr(workspace),
@@ -276,6 +296,8 @@ def astro_chunk_attn_bwd_delta(o, d_o, delta=None, stream=None):
     B, n_q, H, D = o.shape
     if delta is None:
         delta = torch.empty((B, H, n_q), dtype=torch.float32, device=o.device)
+        _used_on(stream, delta)
+    _contiguous(o, d_o, delta)
     _check(lib().astro_chunk_attn_bwd_delta(_ptr(o), _ptr(d_o), B, H, D, n_q, _ptr(delta), _stream(stream)),
            "astro_chunk_attn_bwd_delta")
     return delta
@@ -287,6 +309,8 @@ def astro_chunk_attn_bwd_dq(cache, q, k_chunk, v_chunk, lse, delta, d_o, scale: 
     n_kc = 0 if k_chunk is None else k_chunk.shape[1]
     if dq is None:
         dq = torch.empty_like(q)
+        _used_on(stream, dq)
+    _contiguous(q, k_chunk, v_chunk, lse, delta, d_o, dq)
     st = lib().astro_chunk_attn_bwd_dq(None if cache is None else cache.handle, _ptr(q), _ptr(k_chunk), _ptr(v_chunk),
                                        _ptr(lse), _ptr(delta), _ptr(d_o), B, H, D, n_q, n_kc, float(scale), _ptr(dq),
                                        _stream(stream))
@@ -301,8 +325,11 @@ def astro_chunk_attn_bwd_dkv(q, k_chunk, v_chunk, lse, delta, d_o, scale: float,
     n_kc = k_chunk.shape[1]
     if dk_chunk is None:
         dk_chunk = torch.empty_like(k_chunk)
+        _used_on(stream, dk_chunk)
     if dv_chunk is None:
         dv_chunk = torch.empty_like(v_chunk)
+        _used_on(stream, dv_chunk)
+    _contiguous(q, k_chunk, v_chunk, lse, delta, d_o, dk_chunk, dv_chunk)
     st = lib().astro_chunk_attn_bwd_dkv(_ptr(q), _ptr(k_chunk), _ptr(v_chunk), _ptr(lse), _ptr(delta), _ptr(d_o), B, H,
                                         D, n_q, n_kc, float(scale), _ptr(dk_chunk), _ptr(dv_chunk), _stream(stream))
     _check(st, "astro_chunk_attn_bwd_dkv")
@@ -324,8 +351,8 @@ def astro_nft_loss(v_theta, v_old, v_ref, v_target, r_tilde, beta: float, w_poli
         policy = torch.empty(B, dtype=torch.float32, device=v_theta.device)
         kl = None if v_ref is None else torch.empty(B, dtype=torch.float32, device=v_theta.device)
         g = torch.empty_like(v_theta) if grad else None
-    for t in (v_theta, v_old, v_ref, v_target):
-        assert t is None or t.is_contiguous()
+        _used_on(stream, policy, kl, g)
+    _contiguous(v_theta, v_old, v_ref, v_target, g)
     st = lib().astro_nft_loss(_ptr(v_theta), _ptr(v_old), _ptr(v_ref), _ptr(v_target), _ptr(r_tilde), _ptr(w_policy),
                               _ptr(w_kl), B, elems, float(beta), _ptr(policy), _ptr(kl), _ptr(g), _stream(stream))
     _check(st, "astro_nft_loss")
@@ -343,11 +370,17 @@ def astro_chunk_attn_bwd_static(cache, q, k_chunk, v_chunk, o, lse, d_o, scale: 
     shared array; issue them on one stream."""
     B, n_q, H, D = q.shape
     n_kc = 0 if k_chunk is None else k_chunk.shape[1]
+    _contiguous(q, k_chunk, v_chunk, o, lse, d_o, dq, dk_chunk, dv_chunk)
     st = lib().astro_chunk_attn_bwd_static(None if cache is None else cache.handle, _ptr(q), _ptr(k_chunk),
                                            _ptr(v_chunk), _ptr(o), _ptr(lse), _ptr(d_o), B, H, D, n_q, n_kc,
                                            float(scale), _ptr(dq), _ptr(dk_chunk), _ptr(dv_chunk), _stream(stream))
     _check(st, "astro_chunk_attn_bwd_static")
     return dq, dk_chunk, dv_chunk
+
+
+def astro_debug_forward_safe_only(enable: bool) -> None:
+    """Diagnostic switch: make every later forward run its safe pass only (True) or restore normal operation."""
+    _check(lib().astro_debug_forward_safe_only(1 if enable else 0), "astro_debug_forward_safe_only")
 
 
 def astro_selftest_wait_timeout(stream=None) -> None:

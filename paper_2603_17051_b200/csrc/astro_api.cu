@@ -5,6 +5,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -24,8 +25,11 @@ struct astro_kvcache {
   int win_head;    // ring index (0..L-1) of the oldest window frame
   int win_held;    // frames in the window ring, slots S + (head + i) % L
   int64_t frames_seen;
-  bool maps_ready;
-  CUtensorMap tm_k, tm_v;
+  // Tensor maps of the storage: built once (by create when a driver is present, else by the first attention
+  // call) under a once-flag, read-only afterwards, so attention calls from several threads may share a handle.
+  mutable std::once_flag maps_once;
+  mutable astro_status_t maps_status;
+  mutable CUtensorMap tm_k, tm_v;
 };
 
 namespace astro {
@@ -55,15 +59,19 @@ bool desc_ok(const astro_kvcache_desc_t* d) {
 }
 
 // ---- device / driver helpers -------------------------------------------------------------------
+// Per-device facts are cached in atomics: several host threads may make their first call at the same time,
+// and all of them would store the same value.
+constexpr int kMaxDevices = 64;
+
 astro_status_t check_arch() {
-  static int ok_device[64];
+  static std::atomic<int> ok_device[kMaxDevices];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return ASTRO_ERR_CUDA;
-  if (dev >= 0 && dev < 64 && ok_device[dev]) return ASTRO_OK;
+  if (dev >= 0 && dev < kMaxDevices && ok_device[dev].load(std::memory_order_acquire)) return ASTRO_OK;
   int major = 0;
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ASTRO_ERR_CUDA;
   if (major != 10) return ASTRO_ERR_ARCH;
-  if (dev >= 0 && dev < 64) ok_device[dev] = 1;
+  if (dev >= 0 && dev < kMaxDevices) ok_device[dev].store(1, std::memory_order_release);
   return ASTRO_OK;
 }
 
@@ -108,8 +116,7 @@ astro_status_t make_tmap_user(CUtensorMap* out, const void* base, int head_dim, 
   return make_tmap(out, base, head_dim, n_tok, heads, batch, row * heads, row, row * heads * n_tok);
 }
 
-astro_status_t ensure_cache_maps(astro_kvcache* c) {
-  if (c->maps_ready) return ASTRO_OK;
+astro_status_t build_cache_maps(const astro_kvcache* c) {
   const auto& d = c->d;
   const long long tok = static_cast<long long>(d.sink_frames + d.window_frames) * d.tokens_per_frame;
   const unsigned long long row = static_cast<unsigned long long>(d.head_dim) * 2;
@@ -117,9 +124,12 @@ astro_status_t ensure_cache_maps(astro_kvcache* c) {
                                row * tok * d.heads);
   if (s != ASTRO_OK) return s;
   s = make_tmap(&c->tm_v, c->v, d.head_dim, tok, d.heads, d.cache_batch, row, row * tok, row * tok * d.heads);
-  if (s != ASTRO_OK) return s;
-  c->maps_ready = true;
-  return ASTRO_OK;
+  return s;
+}
+
+astro_status_t cache_maps(const astro_kvcache* c) {
+  std::call_once(c->maps_once, [c] { c->maps_status = build_cache_maps(c); });
+  return c->maps_status;
 }
 
 // Physical token ranges of the held frames, merged where adjacent, followed by the chunk's keys.
@@ -155,12 +165,12 @@ template <typename K> astro_status_t set_smem(K kernel, int bytes) {
              : ASTRO_ERR_CUDA;
 }
 
-template <typename K> astro_status_t set_smem_once(K kernel, int bytes, bool (&done)[64]) {
+template <typename K> astro_status_t set_smem_once(K kernel, int bytes, std::atomic<int> (&done)[kMaxDevices]) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return ASTRO_ERR_CUDA;
-  if (dev >= 0 && dev < 64 && done[dev]) return ASTRO_OK;
-  astro_status_t s = set_smem(kernel, bytes);
-  if (s == ASTRO_OK && dev >= 0 && dev < 64) done[dev] = true;
+  if (dev >= 0 && dev < kMaxDevices && done[dev].load(std::memory_order_acquire)) return ASTRO_OK;
+  astro_status_t s = set_smem(kernel, bytes);   // idempotent: a second thread repeating it does no harm
+  if (s == ASTRO_OK && dev >= 0 && dev < kMaxDevices) done[dev].store(1, std::memory_order_release);
   return s;
 }
 
@@ -187,18 +197,21 @@ astro_status_t check_attn_args(const AttnArgs& a, float scale) {
   return ASTRO_OK;
 }
 
+// 0: fast pass with the safe pass as fallback (normal operation); 1: safe pass only (diagnostics and tests).
+std::atomic<int> g_fwd_safe_only{0};
+
 template <int D>
 astro_status_t launch_fwd(const AttnArgs& a, const __nv_bfloat16* q, const CUtensorMap& tkc, const CUtensorMap& tvc,
                           const CUtensorMap& tkx, const CUtensorMap& tvx, const KeySegs& segs, float scale, void* o,
                           float* lse, cudaStream_t st) {
-  static bool done[64];
+  static std::atomic<int> done[kMaxDevices];
   astro_status_t s = set_smem_once(chunk_attn_fwd_kernel<D>, FwdSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
   const int shared = (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
   dim3 grid((a.n_q + kTile - 1) / kTile, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
   chunk_attn_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kTotal, st>>>(
       q, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared,
-      scale * kLog2e, static_cast<__nv_bfloat16*>(o), lse);
+      scale * kLog2e, g_fwd_safe_only.load(std::memory_order_relaxed), static_cast<__nv_bfloat16*>(o), lse);
   return launch_status();
 }
 
@@ -217,7 +230,7 @@ astro_status_t launch_bwd_dq(const AttnArgs& a, const __nv_bfloat16* q, const CU
                              const CUtensorMap& tvc, const CUtensorMap& tkx, const CUtensorMap& tvx,
                              const KeySegs& segs, float scale, const float* lse, const float* delta, void* dq,
                              cudaStream_t st) {
-  static bool done[64];
+  static std::atomic<int> done[kMaxDevices];
   astro_status_t s = set_smem_once(chunk_attn_bwd_dq_kernel<D>, DqSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
   const int shared = (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
@@ -232,7 +245,7 @@ template <int D>
 astro_status_t launch_bwd_dkv(const AttnArgs& a, const CUtensorMap& tq, const CUtensorMap& tdo,
                               const CUtensorMap& tkc, const CUtensorMap& tvc, float scale, const float* lse,
                               const float* delta, void* dk, void* dv, cudaStream_t st) {
-  static bool done[64];
+  static std::atomic<int> done[kMaxDevices];
   astro_status_t s = set_smem_once(chunk_attn_bwd_dkv_kernel<D>, DkvSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
   dim3 grid_k((a.n_kc + kTile - 1) / kTile, a.heads, a.batch);
@@ -291,7 +304,11 @@ astro_status_t astro_kvcache_create(const astro_kvcache_desc_t* desc, void* k_st
   c->v = v_storage;
   c->sink_held = c->win_head = c->win_held = 0;
   c->frames_seen = 0;
-  c->maps_ready = false;
+  c->maps_status = ASTRO_ERR_CUDA;
+  if (get_encode_fn() != nullptr) {   // a driver is present: build the maps now, so attention calls only read them
+    const astro_status_t ms = cache_maps(c);
+    if (ms != ASTRO_OK) { delete c; return ms; }
+  }
   *out = c;
   return ASTRO_OK;
 }
@@ -431,7 +448,7 @@ astro_status_t astro_chunk_attn_fwd(const astro_kvcache_t* cache, const void* q,
     if ((s = make_tmap_user(&tvc, v_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
   }
   if (have_ctx) {
-    if ((s = ensure_cache_maps(const_cast<astro_kvcache*>(cache))) != ASTRO_OK) return s;
+    if ((s = cache_maps(cache)) != ASTRO_OK) return s;
     tkx = cache->tm_k;
     tvx = cache->tm_v;
   }
@@ -484,7 +501,7 @@ astro_status_t astro_chunk_attn_bwd_dq(const astro_kvcache_t* cache, const void*
     if ((s = make_tmap_user(&tvc, v_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
   }
   if (have_ctx) {
-    if ((s = ensure_cache_maps(const_cast<astro_kvcache*>(cache))) != ASTRO_OK) return s;
+    if ((s = cache_maps(cache)) != ASTRO_OK) return s;
     tkx = cache->tm_k;
     tvx = cache->tm_v;
   }
@@ -574,17 +591,17 @@ astro_status_t astro_nft_loss(const void* v_theta, const void* v_old, const void
 static __device__ __align__(256) float g_bwd_static_delta[ASTRO_BWD_STATIC_MAX_ROWS];
 
 static astro_status_t bwd_static_scratch(float** out) {
-  static float* addr[64];
+  static std::atomic<float*> addr[kMaxDevices];   // every thread that races here stores the same address
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return ASTRO_ERR_CUDA;
-  if (dev < 0 || dev >= 64) return ASTRO_ERR_CUDA;
-  if (!addr[dev]) {
-    float* p = nullptr;
+  if (dev < 0 || dev >= kMaxDevices) return ASTRO_ERR_CUDA;
+  float* p = addr[dev].load(std::memory_order_acquire);
+  if (!p) {
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_bwd_static_delta) != cudaSuccess || !p)
       return ASTRO_ERR_CUDA;
-    addr[dev] = p;
+    addr[dev].store(p, std::memory_order_release);
   }
-  *out = addr[dev];
+  *out = p;
   return ASTRO_OK;
 }
 
@@ -597,6 +614,10 @@ astro_status_t astro_chunk_attn_bwd_static(const astro_kvcache_t* cache, const v
   const AttnArgs a{cache, batch, heads, head_dim, n_q, n_kc};
   astro_status_t s = check_attn_args(a, scale);
   if (s != ASTRO_OK) return s;
+  if (!aligned16(q) || !aligned16(o) || !aligned16(d_o) || !aligned16(dq) ||
+      (reinterpret_cast<uintptr_t>(lse) & 3u) ||
+      (n_kc > 0 && (!aligned16(k_chunk) || !aligned16(v_chunk) || !aligned16(dk_chunk) || !aligned16(dv_chunk))))
+    return ASTRO_ERR_ALIGN;
   if (static_cast<long long>(batch) * heads * n_q > ASTRO_BWD_STATIC_MAX_ROWS) return ASTRO_ERR_CAPACITY;
   s = check_arch();
   if (s != ASTRO_OK) return s;
@@ -609,6 +630,11 @@ astro_status_t astro_chunk_attn_bwd_static(const astro_kvcache_t* cache, const v
   if (s != ASTRO_OK || n_kc == 0) return s;
   return astro_chunk_attn_bwd_dkv(q, k_chunk, v_chunk, lse, delta, d_o, batch, heads, head_dim, n_q, n_kc, scale,
                                   dk_chunk, dv_chunk, stream);
+}
+
+astro_status_t astro_debug_forward_safe_only(int enable) {
+  g_fwd_safe_only.store(enable ? 1 : 0, std::memory_order_relaxed);
+  return ASTRO_OK;
 }
 
 astro_status_t astro_selftest_wait_timeout(void* stream) {

@@ -1,19 +1,26 @@
 // Forward of chunk attention over the rolling cache: O and LSE for one 128-query tile per CTA.
 //
 // Warp-specialised, one CTA per SM:
-//   kFwdGroups softmax groups of 4 warps: group g owns keys [g, g+1) * 128 / kFwdGroups of every key tile,
-//   one query row per thread; then one warp whose first thread issues every tcgen05 MMA, one for TMA loads
+//   two softmax groups of 4 warps: group g owns keys [64 g, 64 g + 64) of every key tile, one query row
+//   per thread; then one warp whose first thread issues every tcgen05 MMA, one for TMA loads
 // Q lives in tensor memory (bf16 pairs, written once by the softmax threads) and is the A operand of
 // S = Q K^T, so shared memory only carries K and V: an MMA with both operands in shared memory reads
 // 128 B/clk, the whole shared-memory bandwidth, and then competes with the TMA writes of the next tiles.
-// S of a whole key tile is one 128x128 MMA into one of two S buffers, issued two tiles ahead.
-// The threads that share a query row (one per group) keep the same reference exponent for the row, so all
-// parts of P V accumulate into ONE O accumulator; each keeps its own partial row sum.  The fast path takes
-// no row maximum: a row re-references itself (true tile maximum, O and row sums rescaled) only when a tile's
-// row sum leaves the safe range.  P is written as bf16 pairs over the thread's own S columns.  K and V tiles
-// travel through 3-deep rings.
-// Part of the exponentials is evaluated by a polynomial on the FMA pipe, because the special-function
-// unit (16 exp2 per clock per SM) is as busy as the tensor core at head_dim 128.
+// S of a whole key tile is one 128x128 MMA into one of two S buffers, issued two tiles ahead.  P is written
+// as bf16 pairs over the thread's own S columns and feeds P V from tensor memory.  K and V tiles travel
+// through 3-deep rings.  Part of the exponentials is evaluated by a polynomial on the FMA pipe, because
+// the special-function unit (16 exp2 per clock per SM) is as busy as the tensor core at head_dim 128.
+//
+// The kernel makes up to two passes over the keys:
+//   fast pass  every row keeps ONE reference exponent, the maximum of its first key tile.  exp2(s - m) is
+//              exact for any reference as long as nothing overflows (bf16 and fp32 share the exponent range,
+//              so later scores may exceed the reference by ~100 in log2 units), so O is never rescaled, the
+//              threads of a row never have to agree on anything after the first tile, and a thread hands
+//              its P to the MMA thread in two halves: P V of the first half runs while the second half is
+//              still being exponentiated.
+//   safe pass  only if some row of the CTA saw a sum beyond 2^100, an infinity or a NaN in the fast pass: the
+//              whole tile is recomputed with a running reference that follows the row maximum (rescaling O
+//              and the row sums when a tile's row sum leaves the safe range).
 //   TMEM columns: S buffers [0,128) [128,256)   O [256,256+D)   Q [384,384+D/2)
 #pragma once
 #include "attn_common.cuh"
@@ -24,68 +31,433 @@ constexpr int kFwdKStages = 3, kFwdVStages = 3, kFwdSBufs = 2;
 constexpr int kFwdGroups = 2;                    // more warps per scheduler hide the exp2 latency
 constexpr int kFwdCols = kTile / kFwdGroups;     // keys per group and tile
 constexpr int kFwdThreads = 128 * kFwdGroups + 64;
+constexpr int kFwdBarSlots = 24;                 // mbarriers of one pass
 
 template <int D> struct FwdSmem {
   static constexpr int kK = 0;
   static constexpr int kV = kK + kFwdKStages * TileGeom<D>::kBytes;
   static constexpr int kMax = kV + kFwdVStages * TileGeom<D>::kBytes;  // float [2 parities + 1][groups][128]
-  static constexpr int kBars = kMax + 3 * kFwdGroups * kTile * 4;
-  static constexpr int kTotal = kBars + 256 + 1024;  // barriers, tmem holder, abort flag + slack to align to 1024
+  static constexpr int kBars = kMax + 3 * kFwdGroups * kTile * 4;      // two sets of barriers, then 3 words
+  static constexpr int kTotal = kBars + 2 * kFwdBarSlots * 8 + 64 + 1024;  // + slack to align to 1024
 };
 
 constexpr int kPolyOf8 = 2;  // of every 8 pairs of exponentials, how many use the polynomial on the FMA pipe
-constexpr float kRowSumLimit = 1073741824.f;  // 2^30: a tile row sum beyond it makes the row re-reference itself
+constexpr float kRowSumLimit = 1073741824.f;        // safe pass: a tile row sum beyond 2^30 re-references the row
+constexpr float kFastSumLimit = 1.2676506e30f;      // fast pass: a row sum beyond 2^100 sends the CTA to the safe pass
+constexpr float kPolyArgLimit = 126.f;              // largest exponent the polynomial exp2 may be handed
+
+// The mbarriers of one pass.  The two passes use separate sets, so a late arrival of the first pass can
+// never land in a phase of the second.
+struct FwdBars {
+  uint64_t *q_full, *k_full, *k_empty, *v_full, *v_empty, *s_full, *p_full, *pv_done, *o_full;
+  __device__ explicit FwdBars(uint64_t* b)
+      : q_full(b), k_full(b + 1), k_empty(k_full + kFwdKStages), v_full(k_empty + kFwdKStages),
+        v_empty(v_full + kFwdVStages), s_full(v_empty + kFwdVStages), p_full(s_full + kFwdSBufs),
+        pv_done(p_full + 2 * kFwdSBufs), o_full(pv_done + 2) {}
+  // p_full: safe pass [group][S buffer], 128 arrivals each (the groups may run up to two tiles ahead of the
+  // MMA thread, so the barriers rotate with the S buffers); fast pass [half][S buffer], 256 arrivals each.
+  __device__ void init(int q_count, int p_count) const {
+    mbar_init(q_full, q_count);
+    for (int i = 0; i < kFwdKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
+    for (int i = 0; i < kFwdVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
+    for (int i = 0; i < kFwdSBufs; ++i) mbar_init(s_full + i, 1);
+    for (int i = 0; i < 2 * kFwdSBufs; ++i) mbar_init(p_full + i, p_count);
+    mbar_init(pv_done, 1);
+    mbar_init(pv_done + 1, 1);
+    mbar_init(o_full, 1);
+  }
+};
+
+// What every role of the CTA needs to know about its work unit.
+template <int D> struct FwdUnit {
+  const CUtensorMap *tm_kc, *tm_vc, *tm_kx, *tm_vx;
+  const KeySegs* segs;
+  uint8_t *sK, *sV;
+  float* smax;
+  volatile int* abort_flag;
+  uint32_t tmem_base;
+  int n_tiles, h, b, bx;
+};
+
+constexpr uint32_t kFwdColS = 0 /* + 128 * buffer */, kFwdColO = 256, kFwdColQ = 384;
+
+// ---------------------------------------------------------------------------------- TMA producer (one thread)
+// K runs ahead of V by the S look-ahead: order the loads K0 K1 | V0 K2 | V1 K3 | ...
+template <int D>
+__device__ __forceinline__ void fwd_produce(const FwdUnit<D>& u, const FwdBars& bar) {
+  const KeySegs& segs = *u.segs;
+  KeyTileIter itk, itv;
+  auto load_k = [&](int j) {
+    const int st = j % kFwdKStages;
+    const bool fc = itk.from_chunk(segs);
+    mbar_wait_spin(bar.k_empty + st, ((j / kFwdKStages) & 1) ^ 1, u.abort_flag);
+    mbar_arrive_expect_tx(bar.k_full + st, TileGeom<D>::kBytes);
+    tma_load_tile<D>(u.sK + st * TileGeom<D>::kBytes, fc ? u.tm_kc : u.tm_kx, bar.k_full + st, itk.row0(segs), u.h,
+                     fc ? u.b : u.bx);
+    itk.next(segs);
+  };
+  auto load_v = [&](int j) {
+    const int st = j % kFwdVStages;
+    const bool fc = itv.from_chunk(segs);
+    mbar_wait_spin(bar.v_empty + st, ((j / kFwdVStages) & 1) ^ 1, u.abort_flag);
+    mbar_arrive_expect_tx(bar.v_full + st, TileGeom<D>::kBytes);
+    tma_load_tile<D>(u.sV + st * TileGeom<D>::kBytes, fc ? u.tm_vc : u.tm_vx, bar.v_full + st, itv.row0(segs), u.h,
+                     fc ? u.b : u.bx);
+    itv.next(segs);
+  };
+  for (int j = 0; j < kFwdSBufs && j < u.n_tiles; ++j) load_k(j);
+  for (int j = 0; j < u.n_tiles; ++j) {
+    load_v(j);
+    if (j + kFwdSBufs < u.n_tiles) load_k(j + kFwdSBufs);
+  }
+}
+
+// ---------------------------------------------------------------------------------- MMA issuer (one thread)
+// kFast: P of a tile arrives in two halves per group (p_full[half][buffer]); the P V MMAs of the first halves
+// are issued as soon as those are there.  Otherwise P arrives per group (p_full[group][buffer]) and every
+// group is awaited first, because any of them may have rescaled its part of O.
+template <int D, bool kFast>
+__device__ __forceinline__ void fwd_issue(const FwdUnit<D>& u, const FwdBars& bar) {
+  const uint64_t k_desc0 = desc_kmajor(smem_u32(u.sK));
+  constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kTile, false, false);
+  constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);
+  const uint32_t tmem_base = u.tmem_base;
+  auto issue_s = [&](int j) {  // S(j) -> buffer j % 2; free because the PV of tile j-2 was issued before
+    const int st = j % kFwdKStages;
+    mbar_wait_spin(bar.k_full + st, (j / kFwdKStages) & 1, u.abort_flag);
+    tc_fence_after_sync();
+    const uint64_t k_desc = desc_step(k_desc0, st * TileGeom<D>::kBytes);
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k)  // 16 elements of the head dimension = 8 packed Q columns
+      mma_ts(tmem_base + kFwdColS + (j % kFwdSBufs) * 128, tmem_base + kFwdColQ + k * 8,
+             desc_step(k_desc, (k >> 2) * TileGeom<D>::kBlockBytes + (k & 3) * 32), idesc_s, k > 0);
+    mma_commit(bar.k_empty + st);
+    mma_commit(bar.s_full + j % kFwdSBufs);
+  };
+  if (kFast) {
+    mbar_wait_spin(bar.q_full, 0, u.abort_flag);
+    tc_fence_after_sync();
+  }
+  for (int j = 0; j < kFwdSBufs && j < u.n_tiles; ++j) issue_s(j);
+  for (int j = 0; j < u.n_tiles; ++j) {
+    const int st = j % kFwdVStages, buf = j % kFwdSBufs;
+    const uint32_t pcol = tmem_base + kFwdColS + buf * 128;
+    const uint64_t v_desc = desc_mnmajor(smem_u32(u.sV + st * TileGeom<D>::kBytes), TileGeom<D>::kBlockBytes);
+    mbar_wait_spin(bar.v_full + st, (j / kFwdVStages) & 1, u.abort_flag);
+    // P of 16 keys = 8 packed columns; group g's pairs start at its own S columns
+    auto pv = [&](int kb, uint32_t accumulate) {
+      const uint32_t a = pcol + (kb * 16 / kFwdCols) * kFwdCols + (kb * 16 % kFwdCols) / 2;
+      mma_ts(tmem_base + kFwdColO, a, desc_step(v_desc, kb * 2048), idesc_pv, accumulate);
+    };
+    if (kFast) {
+      constexpr int kPerHalf = kFwdCols / 32;  // 16-key MMAs per group and half
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        mbar_wait_spin(bar.p_full + half * kFwdSBufs + buf, (j / kFwdSBufs) & 1, u.abort_flag);
+        tc_fence_after_sync();
+#pragma unroll
+        for (int g = 0; g < kFwdGroups; ++g)
+#pragma unroll
+          for (int i = 0; i < kPerHalf; ++i)
+            pv(g * (kFwdCols / 16) + half * kPerHalf + i, (j > 0 || half > 0 || g > 0 || i > 0) ? 1u : 0u);
+      }
+    } else {
+#pragma unroll
+      for (int g = 0; g < kFwdGroups; ++g)
+        mbar_wait_spin(bar.p_full + g * kFwdSBufs + buf, (j / kFwdSBufs) & 1, u.abort_flag);
+      tc_fence_after_sync();
+#pragma unroll
+      for (int kb = 0; kb < kTile / 16; ++kb) pv(kb, (j > 0 || kb > 0) ? 1u : 0u);
+      mma_commit(bar.pv_done + (j & 1));
+    }
+    mma_commit(bar.v_empty + st);
+    if (j + kFwdSBufs < u.n_tiles) issue_s(j + kFwdSBufs);
+  }
+  mma_commit(bar.o_full);
+}
+
+// exp2(s * scale_log2 - m) for 32 consecutive keys of one row, as 16 bf16 pairs; returns their sum.
+// `valid` = how many of the 32 keys exist (the rest get P = 0 whatever their S, which may be stale data).
+// kPolyOf8 of every 8 pairs take the polynomial; the largest argument it was handed is folded into poly_max.
+__device__ __forceinline__ float fwd_exp32(const uint32_t (&s)[32], int valid, float scale_log2, float neg_m,
+                                           uint32_t (&pk)[16], float& poly_max) {
+  if (valid < 32) {
+    float sum = 0.f;
+#pragma unroll
+    for (int c = 0; c < 32; c += 2) {
+      float p0 = fast_exp2(fmaf(__uint_as_float(s[c]), scale_log2, neg_m));
+      float p1 = fast_exp2(fmaf(__uint_as_float(s[c + 1]), scale_log2, neg_m));
+      if (c >= valid) p0 = 0.f;
+      if (c + 1 >= valid) p1 = 0.f;
+      sum += p0 + p1;
+      pk[c >> 1] = pack_bf16(p0, p1);
+    }
+    return sum;
+  }
+  const uint64_t sc2 = f32x2(scale_log2, scale_log2), nm2 = f32x2(neg_m, neg_m);
+  uint64_t acc_a = f32x2(0.f, 0.f), acc_b = f32x2(0.f, 0.f);
+#pragma unroll
+  for (int c = 0; c < 32; c += 2) {
+    const uint64_t x2 = fma2(f32x2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);
+    float p0, p1, x0, x1;
+    f32x2_split(x2, x0, x1);
+    if (((c >> 1) & 7) < kPolyOf8) {
+      poly_max = max3(poly_max, x0, x1);
+      exp2_poly_pair(x2, p0, p1);
+    } else {
+      p0 = fast_exp2(x0);
+      p1 = fast_exp2(x1);
+    }
+    if ((c >> 1) & 1) acc_a = add2(acc_a, f32x2(p0, p1));
+    else acc_b = add2(acc_b, f32x2(p0, p1));
+    pk[c >> 1] = pack_bf16(p0, p1);
+  }
+  float r0, r1;
+  f32x2_split(add2(acc_a, acc_b), r0, r1);
+  return r0 + r1;
+}
+
+// Epilogue shared by both passes: row sum = sum of the groups' partial sums; 32-column slices of the output
+// row are dealt round-robin to the groups.  Returns false if a stored value was not finite.
+template <int D>
+__device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, const FwdBars& bar, int g, int r, uint32_t tmem_lane,
+                                             float m_run, float l_run, bool in_range, __nv_bfloat16* dst,
+                                             float* lse_dst) {
+  mbar_wait(bar.o_full, 0, u.abort_flag);
+  tc_fence_after_sync();
+  float* ex = u.smax;  // free: the last exchange through it was consumed before the last P was published
+  ex[g * kTile + r] = l_run;
+  named_barrier_sync(5, 128 * kFwdGroups);
+  float l = 0.f;
+#pragma unroll
+  for (int og = 0; og < kFwdGroups; ++og) l += ex[og * kTile + r];
+  const float inv_l = 1.f / l;
+  uint32_t worst = 0;
+#pragma unroll
+  for (int c4 = 0; c4 < D / 32; ++c4) {
+    if (c4 % kFwdGroups != g) continue;
+    uint32_t acc[32];
+    tmem_ld32(tmem_lane + kFwdColO + c4 * 32, acc);
+    tmem_wait_ld();
+#pragma unroll
+    for (int c = 0; c < 32; ++c) {
+      acc[c] = __float_as_uint(__uint_as_float(acc[c]) * inv_l);
+      worst = max(worst, acc[c] & 0x7fffffffu);
+    }
+    if (in_range) {
+      uint4* out = reinterpret_cast<uint4*>(dst + c4 * 32);
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        uint4 w;
+        w.x = pack_bf16(__uint_as_float(acc[8 * v + 0]), __uint_as_float(acc[8 * v + 1]));
+        w.y = pack_bf16(__uint_as_float(acc[8 * v + 2]), __uint_as_float(acc[8 * v + 3]));
+        w.z = pack_bf16(__uint_as_float(acc[8 * v + 4]), __uint_as_float(acc[8 * v + 5]));
+        w.w = pack_bf16(__uint_as_float(acc[8 * v + 6]), __uint_as_float(acc[8 * v + 7]));
+        out[v] = w;
+      }
+    }
+  }
+  if (g == 0 && in_range && lse_dst != nullptr) *lse_dst = (m_run + log2f(l)) * 0.6931471805599453f;
+  return worst < 0x7f800000u;
+}
+
+// ---------------------------------------------------------------------------------- softmax, fast pass
+// Returns false if the row must be redone by the safe pass.
+template <int D>
+__device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdBars& bar, int warp, int r,
+                                                 float scale_log2, bool in_range, __nv_bfloat16* dst,
+                                                 float* lse_dst) {
+  const KeySegs& segs = *u.segs;
+  const int g = warp >> 2;
+  const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+  float m_ref = 0.f, l_run = 0.f, poly_max = -INFINITY;
+  int j = 0;
+  for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
+    const int tile_valid = it.valid(segs);
+    const int valid = tile_valid - kFwdCols * g;  // valid keys of this group's share (may be <= 0)
+    const int buf = j % kFwdSBufs;
+    const uint32_t colS = kFwdColS + buf * 128 + g * kFwdCols;
+    mbar_wait(bar.s_full + buf, (j / kFwdSBufs) & 1, u.abort_flag);
+    tc_fence_after_sync();
+    uint32_t s[2][32];
+    tmem_ld32(tmem_lane + colS, s[0]);
+    tmem_ld32(tmem_lane + colS + 32, s[1]);
+    tmem_wait_ld();
+    if (j == 0) {
+      // the row's one reference: the maximum of the first tile, agreed between the two threads of the row
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c2 = 0; c2 < 2; ++c2)
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+          if (c2 * 32 + c < valid) mx = fmaxf(mx, __uint_as_float(s[c2][c]));
+      float* mslot = u.smax + 2 * kFwdGroups * kTile;
+      mslot[g * kTile + r] = mx;
+      named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
+      mx = fmaxf(mx, mslot[(g ^ 1) * kTile + r]);   // finite unless the inputs are not: >= 1 valid key
+      m_ref = mx * scale_log2;
+    }
+    const float neg_m = -m_ref;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      uint32_t pk[16];
+      l_run += fwd_exp32(s[half], valid - 32 * half, scale_log2, neg_m, pk, poly_max);
+      tmem_st16(tmem_lane + colS + half * 16, pk);   // in place: this thread has read all of its S columns
+      if (half == 0 && g == 0 && tile_valid < kTile) {
+        // Rows past the segment's end may hold stale cache contents: P is 0 there, but 0 * NaN is NaN.
+        // Group 0 clears them before publishing its first half, which every PV MMA of the tile is issued after.
+        const int st = j % kFwdVStages;
+        mbar_wait(bar.v_full + st, (j / kFwdVStages) & 1, u.abort_flag);
+        zero_tile_rows_from<D>(u.sV + st * TileGeom<D>::kBytes, tile_valid, r);
+      }
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(bar.p_full + half * kFwdSBufs + buf);
+    }
+  }
+  bool ok = (l_run < kFastSumLimit) && !(poly_max > kPolyArgLimit);   // false for inf and NaN too
+  ok = fwd_epilogue<D>(u, bar, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
+  return ok;
+}
+
+// ---------------------------------------------------------------------------------- softmax, safe pass
+// The threads that share a query row (one per group) keep the same running reference for the row, so all
+// parts of P V accumulate into ONE O accumulator; each keeps its own partial row sum.  No row maximum while
+// nothing happens: a tile is exponentiated against the row's current reference; only when a tile's row sum
+// leaves the safe range (>= 2^30, inf or NaN, or the polynomial was handed an argument beyond its range), or
+// on the first tile, do the two threads agree (one 64-thread named barrier per warp pair and tile carries the
+// decision) to take the tile's true maximum as the new reference, rescaling O and the row sums.
+template <int D>
+__device__ __forceinline__ void fwd_softmax_safe(const FwdUnit<D>& u, const FwdBars& bar, int warp, int r,
+                                                 float scale_log2, bool in_range, __nv_bfloat16* dst,
+                                                 float* lse_dst) {
+  const KeySegs& segs = *u.segs;
+  const int g = warp >> 2;
+  constexpr int NL = kFwdCols / 32;  // 32-column TMEM loads per thread and tile
+  const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+  float m_run = -INFINITY, l_run = 0.f;
+  int j = 0;
+  for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
+    const int tile_valid = it.valid(segs);
+    const int valid = tile_valid - kFwdCols * g;
+    const int buf = j % kFwdSBufs;
+    const uint32_t colS = kFwdColS + buf * 128 + g * kFwdCols;
+    mbar_wait(bar.s_full + buf, (j / kFwdSBufs) & 1, u.abort_flag);
+    tc_fence_after_sync();
+
+    uint32_t pk[NL][16];
+    auto exponentiate = [&](bool& overflow) -> float {
+      uint32_t s[NL][32];
+#pragma unroll
+      for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);
+      tmem_wait_ld();
+      float sum = 0.f, poly_max = -INFINITY;
+#pragma unroll
+      for (int c2 = 0; c2 < NL; ++c2) sum += fwd_exp32(s[c2], valid - 32 * c2, scale_log2, -m_run, pk[c2], poly_max);
+      overflow = !(sum < kRowSumLimit) || poly_max > kPolyArgLimit;   // also true for inf and NaN
+      return sum;
+    };
+
+    float rowsum = 0.f;
+    bool redo = m_run == -INFINITY;
+    if (!__all_sync(0xffffffffu, redo)) {
+      bool overflow;
+      rowsum = exponentiate(overflow);
+      redo = redo || overflow;
+    }
+    float* fslot = u.smax + (j & 1) * kFwdGroups * kTile;
+    fslot[g * kTile + r] = redo ? 1.f : 0.f;
+    named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
+#pragma unroll
+    for (int og = 0; og < kFwdGroups; ++og) redo = redo || fslot[og * kTile + r] != 0.f;
+    float alpha = 1.f;
+    if (__any_sync(0xffffffffu, redo)) {
+      // exact tile maximum, shared between the threads of the row; rows of the warp that did not ask for it
+      // keep their reference
+      uint32_t s[NL][32];
+#pragma unroll
+      for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);   // S is still intact
+      tmem_wait_ld();
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c2 = 0; c2 < NL; ++c2)
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+          if (c2 * 32 + c < valid) mx = fmaxf(mx, __uint_as_float(s[c2][c]));
+      float* mslot = u.smax + 2 * kFwdGroups * kTile;
+      mslot[g * kTile + r] = mx;
+      named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
+#pragma unroll
+      for (int og = 0; og < kFwdGroups; ++og) mx = fmaxf(mx, mslot[og * kTile + r]);  // finite: >= 1 valid key
+      if (redo) {
+        const float m_new = mx * scale_log2;
+        if (m_run != -INFINITY) alpha = fast_exp2(m_run - m_new);   // may be > 1 if the max went down: exact too
+        m_run = m_new;
+      }
+      if (j > 0) {
+        // O must be at rest: wait for the P V of the previous tile.  The barriers alternate with the tile
+        // parity, so the awaited phase is at most one completion away.
+        mbar_wait(bar.pv_done + ((j - 1) & 1), ((j - 1) >> 1) & 1, u.abort_flag);
+        tc_fence_after_sync();
+        // 32-column slices of the row are dealt round-robin to the groups
+#pragma unroll
+        for (int c4 = 0; c4 < D / 32; ++c4) {
+          if (c4 % kFwdGroups != g) continue;
+          uint32_t acc[32];
+          tmem_ld32(tmem_lane + kFwdColO + c4 * 32, acc);
+          tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) acc[c] = __float_as_uint(__uint_as_float(acc[c]) * alpha);
+          tmem_st32(tmem_lane + kFwdColO + c4 * 32, acc);
+        }
+      }
+      l_run *= alpha;
+      bool overflow;
+      rowsum = exponentiate(overflow);
+    }
+    l_run += rowsum;
+#pragma unroll
+    for (int c2 = 0; c2 < NL; ++c2) tmem_st16(tmem_lane + colS + c2 * 16, pk[c2]);
+    if (g == 0 && tile_valid < kTile) {
+      const int st = j % kFwdVStages;
+      mbar_wait(bar.v_full + st, (j / kFwdVStages) & 1, u.abort_flag);
+      zero_tile_rows_from<D>(u.sV + st * TileGeom<D>::kBytes, tile_valid, r);
+    }
+    tmem_wait_st();
+    tc_fence_before_sync();
+    mbar_arrive(bar.p_full + g * kFwdSBufs + buf);
+  }
+  fwd_epilogue<D>(u, bar, g, r, tmem_lane, m_run, l_run, in_range, dst, lse_dst);
+}
 
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant__ CUtensorMap tm_kc,
                       const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kx,
-                      const __grid_constant__ CUtensorMap tm_vx, const KeySegs segs, const int n_q, const int heads,
-                      const int cache_shared, const float scale_log2, __nv_bfloat16* __restrict__ o,
-                      float* __restrict__ lse) {
+                      const __grid_constant__ CUtensorMap tm_vx, const __grid_constant__ KeySegs segs, const int n_q,
+                      const int heads, const int cache_shared, const float scale_log2, const int force_safe,
+                      __nv_bfloat16* __restrict__ o, float* __restrict__ lse) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
-  uint8_t* sK = smem + FwdSmem<D>::kK;
-  uint8_t* sV = smem + FwdSmem<D>::kV;
-  float* smax = reinterpret_cast<float*>(smem + FwdSmem<D>::kMax);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + FwdSmem<D>::kBars);
-  uint64_t* q_full = bars;
-  uint64_t* k_full = bars + 1;                    // [kFwdKStages]
-  uint64_t* k_empty = k_full + kFwdKStages;
-  uint64_t* v_full = k_empty + kFwdKStages;       // [kFwdVStages]
-  uint64_t* v_empty = v_full + kFwdVStages;
-  uint64_t* s_full = v_empty + kFwdVStages;       // [kFwdSBufs]
-  // The groups may run up to two tiles ahead of the MMA thread (S is ready that far), so the P barriers
-  // rotate with the S buffers: a barrier is reused only after the MMA thread has consumed its last phase.
-  uint64_t* p_full = s_full + kFwdSBufs;          // [kFwdGroups][kFwdSBufs]
-  uint64_t* pv_done = p_full + kFwdGroups * kFwdSBufs;  // [2] by tile parity
-  uint64_t* o_full = pv_done + 2;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(o_full + 1);
+  uint64_t* bar_mem = reinterpret_cast<uint64_t*>(smem + FwdSmem<D>::kBars);
+  const FwdBars bar_fast(bar_mem), bar_safe(bar_mem + kFwdBarSlots);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bar_mem + 2 * kFwdBarSlots);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  volatile int* redo_flag = reinterpret_cast<volatile int*>(tmem_holder + 2);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // With one shared cache (frozen prefix of a sample group) the samples of a head are launched next to each
   // other, so the head's cached K/V is fetched from HBM once and served to the whole group out of L2.
   const int q0 = blockIdx.x * kTile;
   const int h = cache_shared ? blockIdx.z : blockIdx.y, b = cache_shared ? blockIdx.y : blockIdx.z;
-  const int bx = cache_shared ? 0 : b;
   constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kColS = 0 /* + 128 * buffer */, kColO = 256, kColQ = 384;
   constexpr int kMmaWarp = 4 * kFwdGroups, kTmaWarp = 4 * kFwdGroups + 1;
-  const int n_tiles = seg_tiles(segs);
 
   if (tid == 0) {
-    mbar_init(q_full, 128 * (D / 64));  // the threads that write Q into tensor memory
-    for (int i = 0; i < kFwdKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
-    for (int i = 0; i < kFwdVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
-    for (int i = 0; i < kFwdSBufs; ++i) {
-      mbar_init(s_full + i, 1);
-      for (int g = 0; g < kFwdGroups; ++g) mbar_init(p_full + g * kFwdSBufs + i, 128);
-    }
-    mbar_init(pv_done, 1);
-    mbar_init(pv_done + 1, 1);
-    mbar_init(o_full, 1);
+    bar_fast.init(128 * (D / 64), 128 * kFwdGroups);  // q_full: the threads that write Q into tensor memory
+    bar_safe.init(1, 128);
     *abort_flag = 0;
+    *redo_flag = force_safe;
     fence_mbar_init();
     fence_proxy_async_smem();
   }
@@ -96,90 +468,33 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem_base = *tmem_holder;
 
+  FwdUnit<D> u;
+  u.tm_kc = &tm_kc; u.tm_vc = &tm_vc; u.tm_kx = &tm_kx; u.tm_vx = &tm_vx;
+  u.segs = &segs;
+  u.sK = smem + FwdSmem<D>::kK;
+  u.sV = smem + FwdSmem<D>::kV;
+  u.smax = reinterpret_cast<float*>(smem + FwdSmem<D>::kMax);
+  u.abort_flag = abort_flag;
+  u.tmem_base = *tmem_holder;
+  u.n_tiles = seg_tiles(segs);
+  u.h = h; u.b = b; u.bx = cache_shared ? 0 : b;
+
+  const int r = tid & 127;           // query row inside the tile = TMEM lane (softmax warps)
+  const int row = q0 + r;
+  const bool in_range = row < n_q;
+  __nv_bfloat16* dst = o + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D;
+  float* lse_dst = lse ? lse + (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0) : nullptr;
+
+  // ---- fast pass
   if (warp == kTmaWarp) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      // K runs ahead of V by the S look-ahead: order the loads K0 K1 | V0 K2 | V1 K3 | ...
-      KeyTileIter itk, itv;
-      auto load_k = [&](int j) {
-        const int st = j % kFwdKStages;
-        const bool fc = itk.from_chunk(segs);
-        mbar_wait_spin(k_empty + st, ((j / kFwdKStages) & 1) ^ 1, abort_flag);
-        mbar_arrive_expect_tx(k_full + st, TileGeom<D>::kBytes);
-        tma_load_tile<D>(sK + st * TileGeom<D>::kBytes, fc ? &tm_kc : &tm_kx, k_full + st, itk.row0(segs), h,
-                         fc ? b : bx);
-        itk.next(segs);
-      };
-      auto load_v = [&](int j) {
-        const int st = j % kFwdVStages;
-        const bool fc = itv.from_chunk(segs);
-        mbar_wait_spin(v_empty + st, ((j / kFwdVStages) & 1) ^ 1, abort_flag);
-        mbar_arrive_expect_tx(v_full + st, TileGeom<D>::kBytes);
-        tma_load_tile<D>(sV + st * TileGeom<D>::kBytes, fc ? &tm_vc : &tm_vx, v_full + st, itv.row0(segs), h,
-                         fc ? b : bx);
-        itv.next(segs);
-      };
-      for (int j = 0; j < kFwdSBufs && j < n_tiles; ++j) load_k(j);
-      for (int j = 0; j < n_tiles; ++j) {
-        load_v(j);
-        if (j + kFwdSBufs < n_tiles) load_k(j + kFwdSBufs);
-      }
-    }
+    if (lane == 0 && !force_safe) fwd_produce<D>(u, bar_fast);
   } else if (warp == kMmaWarp) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint64_t k_desc0 = desc_kmajor(smem_u32(sK));
-      constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kTile, false, false);
-      auto issue_s = [&](int j) {  // S(j) -> buffer j % 2; free because the PV of tile j-2 was issued before
-        const int st = j % kFwdKStages;
-        mbar_wait_spin(k_full + st, (j / kFwdKStages) & 1, abort_flag);
-        tc_fence_after_sync();
-        const uint64_t k_desc = desc_step(k_desc0, st * TileGeom<D>::kBytes);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k)  // 16 elements of the head dimension = 8 packed Q columns
-          mma_ts(tmem_base + kColS + (j % kFwdSBufs) * 128, tmem_base + kColQ + k * 8,
-                 desc_step(k_desc, (k >> 2) * TileGeom<D>::kBlockBytes + (k & 3) * 32), idesc_s, k > 0);
-        mma_commit(k_empty + st);
-        mma_commit(s_full + j % kFwdSBufs);
-      };
-      mbar_wait_spin(q_full, 0, abort_flag);
-      tc_fence_after_sync();
-      for (int j = 0; j < kFwdSBufs && j < n_tiles; ++j) issue_s(j);
-      for (int j = 0; j < n_tiles; ++j) {
-        const int st = j % kFwdVStages, buf = j % kFwdSBufs;
-        const uint32_t vt = smem_u32(sV + st * TileGeom<D>::kBytes);
-        const uint32_t pcol = tmem_base + kColS + buf * 128;
-        mbar_wait_spin(v_full + st, (j / kFwdVStages) & 1, abort_flag);
-        // every group first: any of them may have rescaled its part of O, which all MMAs below accumulate into
-#pragma unroll
-        for (int g = 0; g < kFwdGroups; ++g)
-          mbar_wait_spin(p_full + g * kFwdSBufs + buf, (j / kFwdSBufs) & 1, abort_flag);
-        tc_fence_after_sync();
-        // P of 16 keys = 8 packed columns; group g's pairs start at its own S columns
-        constexpr uint32_t idesc = make_idesc_bf16(kTile, D, false, true);
-        const uint64_t v_desc = desc_mnmajor(vt, TileGeom<D>::kBlockBytes);
-#pragma unroll
-        for (int kb = 0; kb < kTile / 16; ++kb) {
-          const uint32_t a = pcol + (kb * 16 / kFwdCols) * kFwdCols + (kb * 16 % kFwdCols) / 2;
-          mma_ts(tmem_base + kColO, a, desc_step(v_desc, kb * 2048), idesc, (j > 0 || kb > 0) ? 1u : 0u);
-        }
-        mma_commit(pv_done + (j & 1));
-        mma_commit(v_empty + st);
-        if (j + kFwdSBufs < n_tiles) issue_s(j + kFwdSBufs);
-      }
-      mma_commit(o_full);
-    }
+    if (lane == 0 && !force_safe) fwd_issue<D, true>(u, bar_fast);
   } else {
-    // ------------------------------------------------------------------ softmax groups
-    const int g = warp >> 2;           // group: keys kFwdCols * g .. of every tile
-    constexpr int NL = kFwdCols / 32;  // 32-column TMEM loads per thread and tile
-    const int r = tid & 127;           // query row inside the tile = TMEM lane
-    const uint32_t tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-    const int row = q0 + r;
-    const bool in_range = row < n_q;
     // Q row -> tensor memory: 64-element halves of the row (32 packed columns each) are dealt to the groups
+    const int g = warp >> 2;
+    const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
 #pragma unroll
     for (int hq = 0; hq < D / 64; ++hq) {
       if (hq % kFwdGroups != g) continue;
@@ -190,170 +505,31 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
         const uint4 t = in_range ? src[v] : make_uint4(0, 0, 0, 0);
         qr[4 * v] = t.x; qr[4 * v + 1] = t.y; qr[4 * v + 2] = t.z; qr[4 * v + 3] = t.w;
       }
-      tmem_st32(tmem_lane + kColQ + hq * 32, qr);
+      tmem_st32(tmem_lane + kFwdColQ + hq * 32, qr);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(q_full);
+      mbar_arrive(bar_fast.q_full);
     }
-    float m_run = -INFINITY, l_run = 0.f;
-    int j = 0;
-    for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
-      const int tile_valid = it.valid(segs);
-      const int valid = tile_valid - kFwdCols * g;  // valid keys of this group's share (may be <= 0)
-      const int buf = j % kFwdSBufs;
-      const uint32_t colS = kColS + buf * 128 + g * kFwdCols;
-      mbar_wait(s_full + buf, (j / kFwdSBufs) & 1, abort_flag);
-      tc_fence_after_sync();
-
-      // P = exp2(s * scale * log2e - m_run) for this thread's keys, with the row sum; m_run is whatever
-      // reference the row has had so far (any reference is exact as long as nothing overflows)
-      auto exponentiate = [&](uint32_t (&pk)[NL][16]) -> float {
-        uint32_t s[NL][32];
-#pragma unroll
-        for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);
-        tmem_wait_ld();
-        const float neg_m = -m_run;
-        float rowsum;
-        if (valid < kFwdCols) {
-          rowsum = 0.f;
-#pragma unroll
-          for (int c2 = 0; c2 < NL; ++c2)
-#pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              float p0 = fast_exp2(fmaf(__uint_as_float(s[c2][c]), scale_log2, neg_m));
-              float p1 = fast_exp2(fmaf(__uint_as_float(s[c2][c + 1]), scale_log2, neg_m));
-              if (c2 * 32 + c >= valid) p0 = 0.f;
-              if (c2 * 32 + c + 1 >= valid) p1 = 0.f;
-              rowsum += p0 + p1;
-              pk[c2][c >> 1] = pack_bf16(p0, p1);
-            }
-        } else {
-          // full tile: packed fp32 arithmetic; kPolyOf8 of every 8 pairs take the polynomial exp2
-          const uint64_t sc2 = f32x2(scale_log2, scale_log2), nm2 = f32x2(neg_m, neg_m);
-          uint64_t acc_a = f32x2(0.f, 0.f), acc_b = f32x2(0.f, 0.f);
-#pragma unroll
-          for (int c2 = 0; c2 < NL; ++c2)
-#pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              const uint64_t x2 = fma2(f32x2(__uint_as_float(s[c2][c]), __uint_as_float(s[c2][c + 1])), sc2, nm2);
-              float p0, p1;
-              if (((c >> 1) & 7) < kPolyOf8) {
-                exp2_poly_pair(x2, p0, p1);
-              } else {
-                float x0, x1;
-                f32x2_split(x2, x0, x1);
-                p0 = fast_exp2(x0);
-                p1 = fast_exp2(x1);
-              }
-              if ((c >> 1) & 1) acc_a = add2(acc_a, f32x2(p0, p1));
-              else acc_b = add2(acc_b, f32x2(p0, p1));
-              pk[c2][c >> 1] = pack_bf16(p0, p1);
-            }
-          float r0, r1;
-          f32x2_split(add2(acc_a, acc_b), r0, r1);
-          rowsum = r0 + r1;
-        }
-        return rowsum;
-      };
-
-      // Fast path: no row maximum at all.  The tile is exponentiated against the row's current reference;
-      // only if a row sum leaves the safe range (or the row has no reference yet: first tile) does the row take
-      // the true maximum of the tile as its new reference.  The two threads of a row must agree, so each
-      // publishes its decision and reads the other's (one 64-thread barrier per warp pair and tile).
-      uint32_t pk[NL][16];
-      float rowsum = 0.f;
-      bool redo = m_run == -INFINITY;
-      if (!__all_sync(0xffffffffu, redo)) {
-        rowsum = exponentiate(pk);
-        redo = redo || !(rowsum < kRowSumLimit);   // also true for inf and NaN
-      }
-      float* fslot = smax + (j & 1) * kFwdGroups * kTile;
-      fslot[g * kTile + r] = redo ? 1.f : 0.f;
-      named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
-#pragma unroll
-      for (int og = 0; og < kFwdGroups; ++og) redo = redo || fslot[og * kTile + r] != 0.f;
-      float alpha = 1.f;
-      if (__any_sync(0xffffffffu, redo)) {
-        // Slow path (first tile, or scores far above everything seen so far): exact tile maximum, shared
-        // between the threads of the row; rows of the warp that did not ask for it keep their reference.
-        uint32_t s[NL][32];
-#pragma unroll
-        for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);   // S is still intact
-        tmem_wait_ld();
-        float mx = -INFINITY;
-#pragma unroll
-        for (int c2 = 0; c2 < NL; ++c2)
-#pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (c2 * 32 + c < valid) mx = fmaxf(mx, __uint_as_float(s[c2][c]));
-        float* mslot = smax + 2 * kFwdGroups * kTile;
-        mslot[g * kTile + r] = mx;
-        named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
-#pragma unroll
-        for (int og = 0; og < kFwdGroups; ++og) mx = fmaxf(mx, mslot[og * kTile + r]);  // finite: >= 1 valid key
-        if (redo) {
-          const float m_new = mx * scale_log2;
-          if (m_run != -INFINITY) alpha = fast_exp2(m_run - m_new);   // may be > 1 if the max went down: exact too
-          m_run = m_new;
-        }
-        if (j > 0) {
-          // O must be at rest: wait for the P V of the previous tile.  The barriers alternate with the tile
-          // parity, so the awaited phase is at most one completion away.
-          mbar_wait(pv_done + ((j - 1) & 1), ((j - 1) >> 1) & 1, abort_flag);
-          tc_fence_after_sync();
-          // 32-column slices of the row are dealt round-robin to the groups
-#pragma unroll
-          for (int c4 = 0; c4 < D / 32; ++c4) {
-            if (c4 % kFwdGroups != g) continue;
-            uint32_t acc[32];
-            tmem_ld32(tmem_lane + kColO + c4 * 32, acc);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) acc[c] = __float_as_uint(__uint_as_float(acc[c]) * alpha);
-            tmem_st32(tmem_lane + kColO + c4 * 32, acc);
-          }
-        }
-        l_run *= alpha;
-        rowsum = exponentiate(pk);
-      }
-      l_run += rowsum;
-#pragma unroll
-      for (int c2 = 0; c2 < NL; ++c2)   // in place: this thread has read all of its S columns
-        tmem_st16(tmem_lane + colS + c2 * 16, pk[c2]);
-      if (g == 0 && tile_valid < kTile) {
-        // Rows past the segment's end may hold stale cache contents: P is 0 there, but 0 * NaN is NaN.
-        // Group 0 clears them before publishing P_0, which both PV MMAs of the tile are issued after.
-        const int st = j % kFwdVStages;
-        mbar_wait(v_full + st, (j / kFwdVStages) & 1, abort_flag);
-        zero_tile_rows_from<D>(sV + st * TileGeom<D>::kBytes, tile_valid, r);
-      }
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(p_full + g * kFwdSBufs + buf);
-    }
-
-    // ---- epilogue: all groups hold the same running max; row sum = sum of the partial sums;
-    //      32-column slices of the output row are dealt round-robin to the groups
-    mbar_wait(o_full, 0, abort_flag);
-    tc_fence_after_sync();
-    float* ex = smax;  // the last tile's maxima were consumed before its P was published
-    ex[g * kTile + r] = l_run;
-    named_barrier_sync(5, 128 * kFwdGroups);
-    float l = 0.f;
-#pragma unroll
-    for (int og = 0; og < kFwdGroups; ++og) l += ex[og * kTile + r];
-    const float inv_l = 1.f / l;
-    __nv_bfloat16* dst = o + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D;
-#pragma unroll
-    for (int c4 = 0; c4 < D / 32; ++c4)
-      if (c4 % kFwdGroups == g) store_row_from_tmem<32>(tmem_lane + kColO + c4 * 32, inv_l, dst + c4 * 32, in_range);
-    if (g == 0 && in_range && lse != nullptr)
-      lse[(static_cast<size_t>(b) * heads + h) * n_q + row] = (m_run + log2f(l)) * 0.6931471805599453f;
+    if (!force_safe && !fwd_softmax_fast<D>(u, bar_fast, warp, r, scale_log2, in_range, dst, lse_dst)) *redo_flag = 1;
   }
 
+  // ---- safe pass, for the whole CTA, if any of its rows asked for it (every MMA of the fast pass has
+  //      finished by now: the softmax threads waited for the last one before their epilogue)
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
+  tc_fence_after_sync();
+  if (*redo_flag && !*abort_flag) {
+    if (warp == kTmaWarp) {
+      if (lane == 0) fwd_produce<D>(u, bar_safe);
+    } else if (warp == kMmaWarp) {
+      if (lane == 0) fwd_issue<D, false>(u, bar_safe);
+    } else {
+      fwd_softmax_safe<D>(u, bar_safe, warp, r, scale_log2, in_range, dst, lse_dst);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+  }
+  if (warp == kMmaWarp) tmem_dealloc(u.tmem_base, kTmemCols);
 }
 
 }  // namespace astro

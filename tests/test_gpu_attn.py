@@ -33,8 +33,17 @@ def _fill(A, Bc, H, D, T, S, L, held, seed, churn=0):
     return cache, model
 
 
+@pytest.fixture
+def safe_pass_only():
+    """Every forward inside the test runs the kernel's safe pass (running row reference) instead of the fast one."""
+    from paper_2603_17051_b200 import binding as A
+    A.astro_debug_forward_safe_only(True)
+    yield
+    A.astro_debug_forward_safe_only(False)
+
+
 def _run_case(A, B, Bc, H, D, T, S, L, held, n_q, n_kc, seed, churn=0, evict_hole=0, scale=None, bwd=True,
-              o_max_abs=1e-2, o_mean_abs=1e-3):
+              sharp=False):
     scale = 1.0 / np.sqrt(D) if scale is None else scale
     cache, model = _fill(A, Bc, H, D, T, S, L, held, seed, churn)
     if evict_hole:
@@ -49,7 +58,7 @@ def _run_case(A, B, Bc, H, D, T, S, L, held, n_q, n_kc, seed, churn=0, evict_hol
     o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, scale)
     A.astro_last_device_status()
     o_ref, lse_ref = orc.chunk_attn_fwd(qf, kx, vx, kf, vf, scale)
-    check_fwd(o, lse, o_ref, lse_ref, o_max_abs=o_max_abs, o_mean_abs=o_mean_abs)
+    check_fwd(o, lse, o_ref, lse_ref, sharp=sharp)
     if bwd:
         g = A.astro_chunk_attn_bwd(cache, q, kc, vc, o, lse, do, scale)
         A.astro_last_device_status()
@@ -84,7 +93,7 @@ def test_tiny_config_streamed_four_chunks():
         assert np.array_equal(host_bits(ke), mk) and np.array_equal(host_bits(ve), mv)
 
 
-@pytest.mark.parametrize("case", [
+PARITY_CASES = [
     # several tiles with ragged tails everywhere, per-sample caches, wrapped ring
     dict(B=2, Bc=2, H=3, D=128, T=100, S=1, L=5, held=6, n_q=300, n_kc=300, seed=100, churn=2),
     # shared frozen prefix (B_c = 1) broadcast over a group of 3
@@ -101,16 +110,27 @@ def test_tiny_config_streamed_four_chunks():
     dict(B=1, Bc=1, H=1, D=128, T=10, S=4, L=3, held=2, n_q=17, n_kc=5, seed=700),
     # exact multiples of the tile
     dict(B=1, Bc=1, H=2, D=128, T=128, S=1, L=3, held=4, n_q=256, n_kc=256, seed=800, churn=1),
-    # a scale other than 1/sqrt(D): near one-hot softmax, the running max moves.  O is then about one V row
-    # (|v| up to ~4.5), so the bf16 rounding of P (2^-9 relative) and of O (half an ulp, 2^-9 |o|) bound the
-    # error by 2^-8 max|v| = 1.8e-2 rather than by the 1e-2 of the 1/sqrt(D) workloads; the mean error of
-    # rounding a unit-magnitude output to bf16 alone is about a quarter ulp, 2^-9.5 E|o| = 1.1e-3, so 2.5e-3.
-    dict(B=1, Bc=1, H=2, D=128, T=64, S=0, L=6, held=6, n_q=200, n_kc=100, seed=900, scale=0.7, o_max_abs=1.8e-2,
-         o_mean_abs=2.5e-3),
-])
+    # a scale other than 1/sqrt(D): near one-hot softmax.  O is then about one V row (|v| up to ~4.5), and the
+    # rounding of the bf16 output alone (half an ulp, up to 7.8e-3 at |o| >= 4) leaves no room inside a flat
+    # 1e-2, so each element is held to 1e-2 + half a bf16 ulp of its reference value (helpers.check_fwd)
+    dict(B=1, Bc=1, H=2, D=128, T=64, S=0, L=6, held=6, n_q=200, n_kc=100, seed=900, scale=0.7, sharp=True),
+    # head_dim 64 with 3 query tiles and 12 key tiles over three segments (wrapped ring + chunk): the 3-deep
+    # K and V rings and the two S buffers wrap several times
+    dict(B=2, Bc=2, H=2, D=64, T=96, S=2, L=8, held=10, n_q=300, n_kc=290, seed=950, churn=3),
+]
+
+
+@pytest.mark.parametrize("case", PARITY_CASES)
 def test_parity_cases(case):
     from paper_2603_17051_b200 import binding as A
     _run_case(A, **case)
+
+
+@pytest.mark.parametrize("case", PARITY_CASES)
+def test_parity_cases_safe_pass(case, safe_pass_only):
+    """The same cases through the forward's safe pass (running row reference, O rescaled on the way)."""
+    from paper_2603_17051_b200 import binding as A
+    _run_case(A, bwd=False, **case)
 
 
 def test_single_key_and_identical_keys_closed_forms_on_gpu():
@@ -313,23 +333,35 @@ def test_random_shapes_and_cache_histories(seed):
     churn = int(rng.integers(0, 4))
     hole = int(rng.integers(0, 2)) if held > S else 0
     scale = float(rng.choice([1.0 / np.sqrt(D), 0.05, 0.3]))
-    loose = scale > 0.2          # sharper softmax: outputs of magnitude ~|v| (see the scale 0.7 case above)
+    sharp = scale > 0.2          # sharper softmax: outputs of magnitude ~|v| (see the scale 0.7 case above)
     _run_case(A, B, Bc, H, D, T, S, L, held, n_q, n_kc, 20000 + 100 * seed, churn=churn, evict_hole=hole, scale=scale,
-              o_max_abs=1.8e-2 if loose else 1e-2, o_mean_abs=2.5e-3 if loose else 1e-3)
+              sharp=sharp)
 
 
-@pytest.mark.parametrize("order", ["rising", "falling", "spike"])
-def test_row_reference_follows_score_jumps_between_tiles(order):
-    """The forward takes no row maximum on its fast path: a row re-references itself only when a tile's row sum
-    leaves the safe range.  Here later key tiles score far above (or below) earlier ones, so that path runs
-    several times per row (rising), never after the first tile (falling), or once in the middle (spike)."""
+@pytest.mark.parametrize("mode", ["normal", "safe_pass"])
+@pytest.mark.parametrize("order", ["rising", "falling", "spike", "steep"])
+def test_row_reference_follows_score_jumps_between_tiles(order, mode):
+    """Later key tiles score far above (or below) earlier ones.  The fast pass keeps the first tile's maximum as
+    the row's reference, which stays exact while exp2 of the difference fits fp32 ("rising", "falling", "spike":
+    differences of tens of nats); "steep" rises by hundreds of nats, the row sums overflow and the kernel repeats
+    the tile in its safe pass.  In the safe pass a row re-references itself whenever a tile's row sum leaves the
+    safe range: several times per row (rising, steep), never after the first tile (falling), once (spike)."""
     from paper_2603_17051_b200 import binding as A
+    A.astro_debug_forward_safe_only(mode == "safe_pass")
+    try:
+        _score_jump_case(A, order)
+    finally:
+        A.astro_debug_forward_safe_only(False)
+
+
+def _score_jump_case(A, order):
     B, H, D, n_q, n_k = 1, 2, 128, 200, 128 * 6 + 40
     qb = synth.normal_bf16(4101, (B, n_q, H, D)); kb = synth.normal_bf16(4102, (B, n_k, H, D))
     vb = synth.normal_bf16(4103, (B, n_k, H, D)); dob = synth.normal_bf16(4104, (B, n_q, H, D))
     kf = orc.bf16_bits_to_f64(kb)
     tile = np.arange(n_k) // 128
-    gain = {"rising": 1.0 + 1.5 * tile, "falling": 10.0 - 1.5 * tile, "spike": np.where(tile == 3, 12.0, 1.0)}[order]
+    gain = {"rising": 1.0 + 1.5 * tile, "falling": 10.0 - 1.5 * tile, "spike": np.where(tile == 3, 12.0, 1.0),
+            "steep": 1.0 + 12.0 * tile}[order]
     kb = synth.f32_to_bf16_bits((kf * gain[None, :, None, None]).astype(np.float32))   # exact in bf16? re-round
     kf = orc.bf16_bits_to_f64(kb)
     q, k, v, do = (dev_bf16(x) for x in (qb, kb, vb, dob))
@@ -339,9 +371,39 @@ def test_row_reference_follows_score_jumps_between_tiles(order):
     A.astro_last_device_status()
     o_ref, lse_ref = orc.chunk_attn_fwd(qf, None, None, kf, vf, scale)
     # near one-hot rows: the output is about one V row, tolerance as in the sharp-softmax case above
-    check_fwd(o, lse, o_ref, lse_ref, o_max_abs=1.8e-2, o_mean_abs=2.5e-3)
+    check_fwd(o, lse, o_ref, lse_ref, sharp=True)
+    if order != "steep":   # keys 73 times the unit scale are a forward case: bf16 dS then carries ~1.1e-2 into dQ
+        g = A.astro_chunk_attn_bwd(None, q, k, v, o, lse, do, scale)
+        check_grads(g, orc.chunk_attn_bwd(qf, None, None, kf, vf, dof, scale))
+
+
+@pytest.mark.parametrize("column", [1, 5, 64 + 2, 64 + 37])
+def test_lone_key_far_above_the_first_tile(column):
+    """No context; one key of the third tile scores about 100 nats above everything before it, all other keys
+    stay near zero.  The key sits on a column whose exponential is taken by the polynomial (column % 16 < 4) or
+    by the special-function unit: either way exp2 of the difference to the row's first reference overflows, which
+    must be noticed (not wrapped into a small number) and the tile redone with a running reference.  The output
+    is then that key's V row and LSE its score."""
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, n_q, n_k = 1, 2, 128, 140, 128 * 3 + 17
+    star = 2 * 128 + column
+    rng_q = orc.bf16_bits_to_f64(synth.normal_bf16(4201, (B, n_q, H, D)))
+    qb = synth.f32_to_bf16_bits((1.0 + 0.25 * rng_q).astype(np.float32))          # a common direction + noise
+    kf = 0.05 * orc.bf16_bits_to_f64(synth.normal_bf16(4202, (B, n_k, H, D)))
+    kf[:, star] = 9.0                                                              # score ~ 9 * 128 / sqrt(128) = 102
+    kb = synth.f32_to_bf16_bits(kf.astype(np.float32))
+    vb = synth.normal_bf16(4203, (B, n_k, H, D)); dob = synth.normal_bf16(4204, (B, n_q, H, D))
+    q, k, v, do = (dev_bf16(x) for x in (qb, kb, vb, dob))
+    qf, kf, vf, dof = (orc.bf16_bits_to_f64(x) for x in (qb, kb, vb, dob))
+    scale = 1.0 / np.sqrt(D)
+    o, lse = A.astro_chunk_attn_fwd(None, q, k, v, scale)
+    A.astro_last_device_status()
+    o_ref, lse_ref = orc.chunk_attn_fwd(qf, None, None, kf, vf, scale)
+    assert lse_ref.min() > 80.0                                                    # the case is what it claims
+    check_fwd(o, lse, o_ref, lse_ref, sharp=True)
+    # one-hot rows: dQ and dK vanish (1e-36) and only rounding noise is left of them; dV is the sum of dO at the key
     g = A.astro_chunk_attn_bwd(None, q, k, v, o, lse, do, scale)
-    check_grads(g, orc.chunk_attn_bwd(qf, None, None, kf, vf, dof, scale))
+    check_grads((None, None, g[2]), orc.chunk_attn_bwd(qf, None, None, kf, vf, dof, scale))
 
 
 def test_calls_follow_the_callers_stream():
