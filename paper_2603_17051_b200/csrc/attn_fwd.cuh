@@ -113,65 +113,60 @@ __device__ __forceinline__ void fwd_produce(const FwdUnit<D>& u, const FwdBars& 
 }
 
 // ---------------------------------------------------------------------------------- MMA issuer (one thread)
-// kFast: P of a tile arrives in two halves per group (p_full[half][buffer]); the P V MMAs of the first halves
-// are issued as soon as those are there.  Otherwise P arrives per group (p_full[group][buffer]) and every
-// group is awaited first, because any of them may have rescaled its part of O.
+// The tensor pipe runs only while this thread keeps handing it MMAs (an issue blocks for about as long as an MMA
+// executes, the queue behind it is short), so every clock this thread spends on anything else is an idle clock of
+// the pipe.  Per key tile it therefore first makes sure of everything the tile needs (V(j), K(j+2), P(j)), then
+// issues P V of tile j and S of tile j+2 as one uninterrupted burst of 16 MMAs, then commits.
+// kFast: P of a tile arrives in two halves per group (p_full[half][buffer]).  Otherwise P arrives per group
+// (p_full[group][buffer]); any of the groups may have rescaled its part of O before it published.
 template <int D, bool kFast>
 __device__ __forceinline__ void fwd_issue(const FwdUnit<D>& u, const FwdBars& bar) {
   const uint64_t k_desc0 = desc_kmajor(smem_u32(u.sK));
   constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kTile, false, false);
   constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);
   const uint32_t tmem_base = u.tmem_base;
+  auto wait_k = [&](int j) {
+    mbar_wait_spin(bar.k_full + j % kFwdKStages, (j / kFwdKStages) & 1, u.abort_flag);
+  };
   auto issue_s = [&](int j) {  // S(j) -> buffer j % 2; free because the PV of tile j-2 was issued before
-    const int st = j % kFwdKStages;
-    mbar_wait_spin(bar.k_full + st, (j / kFwdKStages) & 1, u.abort_flag);
-    tc_fence_after_sync();
-    const uint64_t k_desc = desc_step(k_desc0, st * TileGeom<D>::kBytes);
+    const uint64_t k_desc = desc_step(k_desc0, (j % kFwdKStages) * TileGeom<D>::kBytes);
 #pragma unroll
     for (int k = 0; k < D / 16; ++k)  // 16 elements of the head dimension = 8 packed Q columns
       mma_ts(tmem_base + kFwdColS + (j % kFwdSBufs) * 128, tmem_base + kFwdColQ + k * 8,
              desc_step(k_desc, (k >> 2) * TileGeom<D>::kBlockBytes + (k & 3) * 32), idesc_s, k > 0);
-    mma_commit(bar.k_empty + st);
+  };
+  auto commit_s = [&](int j) {
+    mma_commit(bar.k_empty + j % kFwdKStages);
     mma_commit(bar.s_full + j % kFwdSBufs);
   };
-  if (kFast) {
-    mbar_wait_spin(bar.q_full, 0, u.abort_flag);
+  if (kFast) mbar_wait_spin(bar.q_full, 0, u.abort_flag);
+  for (int j = 0; j < kFwdSBufs && j < u.n_tiles; ++j) {
+    wait_k(j);
     tc_fence_after_sync();
+    issue_s(j);
+    commit_s(j);
   }
-  for (int j = 0; j < kFwdSBufs && j < u.n_tiles; ++j) issue_s(j);
   for (int j = 0; j < u.n_tiles; ++j) {
     const int st = j % kFwdVStages, buf = j % kFwdSBufs;
+    const bool more = j + kFwdSBufs < u.n_tiles;
     const uint32_t pcol = tmem_base + kFwdColS + buf * 128;
     const uint64_t v_desc = desc_mnmajor(smem_u32(u.sV + st * TileGeom<D>::kBytes), TileGeom<D>::kBlockBytes);
     mbar_wait_spin(bar.v_full + st, (j / kFwdVStages) & 1, u.abort_flag);
-    // P of 16 keys = 8 packed columns; group g's pairs start at its own S columns
-    auto pv = [&](int kb, uint32_t accumulate) {
+    if (more) wait_k(j + kFwdSBufs);
+#pragma unroll
+    for (int i = 0; i < 2; ++i)   // halves (fast pass) or groups (safe pass)
+      mbar_wait_spin(bar.p_full + i * kFwdSBufs + buf, (j / kFwdSBufs) & 1, u.abort_flag);
+    tc_fence_after_sync();
+#pragma unroll
+    for (int kb = 0; kb < kTile / 16; ++kb) {
+      // P of 16 keys = 8 packed columns; group g's pairs start at its own S columns
       const uint32_t a = pcol + (kb * 16 / kFwdCols) * kFwdCols + (kb * 16 % kFwdCols) / 2;
-      mma_ts(tmem_base + kFwdColO, a, desc_step(v_desc, kb * 2048), idesc_pv, accumulate);
-    };
-    if (kFast) {
-      constexpr int kPerHalf = kFwdCols / 32;  // 16-key MMAs per group and half
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        mbar_wait_spin(bar.p_full + half * kFwdSBufs + buf, (j / kFwdSBufs) & 1, u.abort_flag);
-        tc_fence_after_sync();
-#pragma unroll
-        for (int g = 0; g < kFwdGroups; ++g)
-#pragma unroll
-          for (int i = 0; i < kPerHalf; ++i)
-            pv(g * (kFwdCols / 16) + half * kPerHalf + i, (j > 0 || half > 0 || g > 0 || i > 0) ? 1u : 0u);
-      }
-    } else {
-#pragma unroll
-      for (int g = 0; g < kFwdGroups; ++g)
-        mbar_wait_spin(bar.p_full + g * kFwdSBufs + buf, (j / kFwdSBufs) & 1, u.abort_flag);
-      tc_fence_after_sync();
-#pragma unroll
-      for (int kb = 0; kb < kTile / 16; ++kb) pv(kb, (j > 0 || kb > 0) ? 1u : 0u);
-      mma_commit(bar.pv_done + (j & 1));
+      mma_ts(tmem_base + kFwdColO, a, desc_step(v_desc, kb * 2048), idesc_pv, (j > 0 || kb > 0) ? 1u : 0u);
     }
+    if (more) issue_s(j + kFwdSBufs);
+    if (!kFast) mma_commit(bar.pv_done + (j & 1));   // tracks the S MMAs too: they are long done when O is needed
     mma_commit(bar.v_empty + st);
-    if (j + kFwdSBufs < u.n_tiles) issue_s(j + kFwdSBufs);
+    if (more) commit_s(j + kFwdSBufs);
   }
   mma_commit(bar.o_full);
 }
