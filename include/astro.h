@@ -10,8 +10,13 @@
  *     keeps alive; the library frees none of it.  The cache handle owns only
  *     host-side metadata.  Query outputs (int*, int64_t*) are HOST pointers.
  *   - Work is enqueued on the given CUDA stream (passed as void*, a cudaStream_t)
- *     and the call returns without synchronising.  Calls on one cache must come
- *     from one host thread; metadata changes take effect in call order.
+ *     and the call returns without synchronising.  Metadata changes take effect in
+ *     call order.  Threads: calls that change a cache (append, evict, reset,
+ *     set_state, destroy) must not run at the same time as any other call on that
+ *     cache; calls that take it as const (the attention calls, query, get_state,
+ *     key_segments, export) may be issued by several host threads at once on one
+ *     handle -- the G candidates of a group decoding against one shared prefix --
+ *     each with its own stream and output buffers.
  *   - bf16 tensors Q, O, K_chunk, V_chunk, dO, dQ, dK_chunk, dV_chunk are
  *     contiguous [batch, tokens, heads, head_dim].  LSE and delta are fp32
  *     [batch, heads, tokens].  Data pointers must be 16-byte aligned.
@@ -60,7 +65,8 @@ size_t astro_kvcache_storage_bytes(const astro_kvcache_desc_t* desc);
  * so that resident KV memory is constant however long the video grows.
  * k_storage/v_storage: device, >= bytes_each each, 16-byte aligned; the layout
  * inside is private ([B_c, H, slot, T, D]).  The storage need not be initialised.
- * The cache starts empty.  *out receives the handle. */
+ * The cache starts empty.  *out receives the handle.  The call also encodes the
+ * tensor maps of the storage (a host-only driver call; nothing is launched). */
 astro_status_t astro_kvcache_create(const astro_kvcache_desc_t* desc, void* k_storage, void* v_storage,
                                     size_t bytes_each, astro_kvcache_t** out);
 
@@ -116,9 +122,9 @@ astro_status_t astro_kvcache_key_segments(const astro_kvcache_t* cache, int n_kc
  * window oldest to newest) to k_out, v_out: device bf16 [B_c, held*T, H, D]. */
 astro_status_t astro_kvcache_export(const astro_kvcache_t* cache, void* k_out, void* v_out, void* stream);
 
-/* Sec. 3.2 (the model "attends exclusively to the KV cache of C_n" while it
- * generates the next clip; G candidates decode against one shared prefix) --
- * forward of chunk attention.  For every sample b, head h and chunk query i:
+/* Sec. 3.2 (while the next clip is generated, attention is restricted to the cached
+ * keys and values of the context C_n; G candidates decode against one shared prefix)
+ * -- forward of chunk attention.  For every sample b, head h and chunk query i:
  *   keys/values = every token held in the cache (of sample b, or of the single
  *   shared cache when B_c = 1) followed by the n_kc chunk tokens;
  *   s_ij = scale * q_i . k_j;  LSE_i = ln sum_j exp(s_ij);  o_i = sum_j exp(s_ij - LSE_i) v_j.
@@ -219,11 +225,17 @@ astro_status_t astro_selftest_wait_timeout(void* stream);
 
 /* Diagnostic switch (the paper has no counterpart).  The forward kernel first runs a fast pass in which a
  * query row keeps the maximum of its first key tile as its one reference exponent, and repeats a 128-query
- * tile with a running reference (the "safe pass") only if a row sum left the range fp32 can hold.  enable != 0
- * makes every later astro_chunk_attn_fwd of this process run the safe pass only; 0 restores normal operation.
- * Results agree within the rounding of bf16 either way; the switch exists so that tests can cover the safe
- * pass on ordinary inputs.  Process-wide, not stream-ordered: it applies to calls made after it returns. */
-astro_status_t astro_debug_forward_safe_only(int enable);
+ * tile with a running reference (the "safe pass") only if a row sum left the range fp32 can hold.
+ *   mode 0  normal operation;
+ *   mode 1  every later astro_chunk_attn_fwd of this process runs the safe pass only;
+ *   mode 2  head_dim 128 calls run the CTA-pair kernel (two query tiles share every K/V tile through one
+ *           tcgen05 cta_group::2 MMA); it has no safe pass of its own: a call whose rows would need one leaves
+ *           a flag that astro_debug_pair_flag reads (and clears) after synchronising the device.
+ * Results agree within the rounding of bf16 in every mode; the switch exists so that tests and benchmarks can
+ * reach each code path on ordinary inputs.  Process-wide, not stream-ordered: it applies to calls made after it
+ * returns.  ASTRO_ERR_SHAPE for any other mode. */
+astro_status_t astro_debug_forward_mode(int mode);
+astro_status_t astro_debug_pair_flag(int* flag);
 
 /* Static, never null. */
 const char* astro_status_string(astro_status_t status);

@@ -20,7 +20,7 @@ EXPORTED = ("astro_kvcache_key_segments", "astro_selftest_wait_timeout", "astro_
             "astro_kvcache_append", "astro_kvcache_evict", "astro_kvcache_query", "astro_kvcache_export",
             "astro_chunk_attn_fwd", "astro_chunk_attn_bwd_workspace_bytes", "astro_chunk_attn_bwd",
             "astro_chunk_attn_bwd_delta", "astro_chunk_attn_bwd_dq", "astro_chunk_attn_bwd_dkv",
-            "astro_chunk_attn_bwd_static", "astro_debug_forward_safe_only",
+            "astro_chunk_attn_bwd_static", "astro_debug_forward_mode", "astro_debug_pair_flag",
             "astro_last_device_status", "astro_status_string")
 
 
@@ -90,8 +90,10 @@ def lib():
     L.astro_chunk_attn_bwd_static.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, vp, vp, vp, vp]
     L.astro_nft_loss.restype = ci
     L.astro_nft_loss.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, C.c_longlong, cf, vp, vp, vp, vp]
-    L.astro_debug_forward_safe_only.restype = ci
-    L.astro_debug_forward_safe_only.argtypes = [ci]
+    L.astro_debug_forward_mode.restype = ci
+    L.astro_debug_forward_mode.argtypes = [ci]
+    L.astro_debug_pair_flag.restype = ci
+    L.astro_debug_pair_flag.argtypes = [C.POINTER(ci)]
     L.astro_selftest_wait_timeout.restype = ci
     L.astro_selftest_wait_timeout.argtypes = [vp]
     L.astro_last_device_status.restype = ci
@@ -378,9 +380,20 @@ def astro_chunk_attn_bwd_static(cache, q, k_chunk, v_chunk, o, lse, d_o, scale: 
     return dq, dk_chunk, dv_chunk
 
 
-def astro_debug_forward_safe_only(enable: bool) -> None:
-    """Diagnostic switch: make every later forward run its safe pass only (True) or restore normal operation."""
-    _check(lib().astro_debug_forward_safe_only(1 if enable else 0), "astro_debug_forward_safe_only")
+FWD_MODE_NORMAL, FWD_MODE_SAFE_ONLY, FWD_MODE_PAIR = 0, 1, 2
+
+
+def astro_debug_forward_mode(mode: int) -> None:
+    """Diagnostic switch: 0 normal operation, 1 every later forward runs its safe pass only, 2 head_dim 128
+    forwards run the CTA-pair kernel."""
+    _check(lib().astro_debug_forward_mode(int(mode)), "astro_debug_forward_mode")
+
+
+def astro_debug_pair_flag() -> int:
+    """Synchronises; 1 if a CTA-pair forward since the last call had a row that needs the safe pass (cleared)."""
+    f = C.c_int()
+    _check(lib().astro_debug_pair_flag(C.byref(f)), "astro_debug_pair_flag")
+    return f.value
 
 
 def astro_selftest_wait_timeout(stream=None) -> None:

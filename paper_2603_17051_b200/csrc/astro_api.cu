@@ -12,6 +12,7 @@
 
 #include "attn_bwd.cuh"
 #include "attn_fwd.cuh"
+#include "attn_fwd_pair.cuh"
 #include "kv_ring.cuh"
 #include "nft_loss.cuh"
 
@@ -96,13 +97,13 @@ encode_tiled_fn get_encode_fn() {
 // swizzle, zero fill outside the tensor.
 astro_status_t make_tmap(CUtensorMap* out, const void* base, int head_dim, long long n_tok, int heads, int batch,
                          unsigned long long stride_tok, unsigned long long stride_head,
-                         unsigned long long stride_batch) {
+                         unsigned long long stride_batch, int box_rows = kTile) {
   encode_tiled_fn fn = get_encode_fn();
   if (!fn) return ASTRO_ERR_CUDA;
   cuuint64_t dims[4] = {static_cast<cuuint64_t>(head_dim), static_cast<cuuint64_t>(n_tok),
                         static_cast<cuuint64_t>(heads), static_cast<cuuint64_t>(batch)};
   cuuint64_t strides[3] = {stride_tok, stride_head, stride_batch};
-  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(kTile), 1, 1};
+  cuuint32_t box[4] = {64, static_cast<cuuint32_t>(box_rows), 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -111,9 +112,20 @@ astro_status_t make_tmap(CUtensorMap* out, const void* base, int head_dim, long 
 }
 
 // Caller tensor [batch, n_tok, H, D].
-astro_status_t make_tmap_user(CUtensorMap* out, const void* base, int head_dim, int n_tok, int heads, int batch) {
+astro_status_t make_tmap_user(CUtensorMap* out, const void* base, int head_dim, int n_tok, int heads, int batch,
+                              int box_rows = kTile) {
   const unsigned long long row = static_cast<unsigned long long>(head_dim) * 2;
-  return make_tmap(out, base, head_dim, n_tok, heads, batch, row * heads, row, row * heads * n_tok);
+  return make_tmap(out, base, head_dim, n_tok, heads, batch, row * heads, row, row * heads * n_tok, box_rows);
+}
+
+// Cache storage seen up to token `end_tok` only (rows from there on read as zeros), box of `box_rows` tokens.
+astro_status_t make_tmap_cache_range(CUtensorMap* out, const astro_kvcache* c, const void* base, long long end_tok,
+                                     int box_rows) {
+  const auto& d = c->d;
+  const long long tok = static_cast<long long>(d.sink_frames + d.window_frames) * d.tokens_per_frame;
+  const unsigned long long row = static_cast<unsigned long long>(d.head_dim) * 2;
+  return make_tmap(out, base, d.head_dim, end_tok, d.heads, d.cache_batch, row, row * tok, row * tok * d.heads,
+                   box_rows);
 }
 
 astro_status_t build_cache_maps(const astro_kvcache* c) {
@@ -197,8 +209,45 @@ astro_status_t check_attn_args(const AttnArgs& a, float scale) {
   return ASTRO_OK;
 }
 
-// 0: fast pass with the safe pass as fallback (normal operation); 1: safe pass only (diagnostics and tests).
-std::atomic<int> g_fwd_safe_only{0};
+// 0: fast pass with the safe pass as fallback (normal operation); 1: safe pass only; 2: CTA-pair kernel where the
+// shape allows it (head_dim 128).  Diagnostics and tests.
+std::atomic<int> g_fwd_mode{0};
+
+// Set by the CTA-pair kernel when a row needs the running-reference pass; read back by astro_debug_pair_flag.
+__device__ int g_pair_needs_safe = 0;
+
+astro_status_t launch_fwd_pair(const AttnArgs& a, const astro_kvcache* cache, bool have_ctx, const void* q,
+                               const void* k_chunk, const void* v_chunk, const KeySegs& segs, float scale, void* o,
+                               float* lse, cudaStream_t st) {
+  static std::atomic<int> done[kMaxDevices];
+  astro_status_t s = set_smem_once(chunk_attn_fwd_pair_kernel, PairSmem::kTotal, done);
+  if (s != ASTRO_OK) return s;
+  PairMaps maps;
+  std::memset(&maps, 0, sizeof(maps));
+  if (a.n_kc > 0) {
+    if ((s = make_tmap_user(&maps.kc, k_chunk, 128, a.n_kc, a.heads, a.batch, 64)) != ASTRO_OK) return s;
+    if ((s = make_tmap_user(&maps.vc, v_chunk, 128, a.n_kc, a.heads, a.batch)) != ASTRO_OK) return s;
+  }
+  if (have_ctx) {
+    int ci = 0;
+    for (int i = 0; i < segs.n; ++i) {
+      if (segs.from_chunk[i]) continue;
+      const long long end = static_cast<long long>(segs.start[i]) + segs.count[i];
+      if ((s = make_tmap_cache_range(&maps.kx[ci], cache, cache->k, end, 64)) != ASTRO_OK) return s;
+      if ((s = make_tmap_cache_range(&maps.vx[ci], cache, cache->v, end, kTile)) != ASTRO_OK) return s;
+      ++ci;
+    }
+  }
+  int* flag = nullptr;
+  if (cudaGetSymbolAddress(reinterpret_cast<void**>(&flag), g_pair_needs_safe) != cudaSuccess) return ASTRO_ERR_CUDA;
+  const int shared = (cache && cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
+  const int tiles = (a.n_q + kTile - 1) / kTile;
+  dim3 grid((tiles + 1) / 2 * 2, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
+  chunk_attn_fwd_pair_kernel<<<grid, kFwdThreads, PairSmem::kTotal, st>>>(
+      static_cast<const __nv_bfloat16*>(q), maps, segs, a.n_q, a.heads, shared, scale * kLog2e,
+      static_cast<__nv_bfloat16*>(o), lse, flag);
+  return launch_status();
+}
 
 template <int D>
 astro_status_t launch_fwd(const AttnArgs& a, const __nv_bfloat16* q, const CUtensorMap& tkc, const CUtensorMap& tvc,
@@ -211,7 +260,7 @@ astro_status_t launch_fwd(const AttnArgs& a, const __nv_bfloat16* q, const CUten
   dim3 grid((a.n_q + kTile - 1) / kTile, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
   chunk_attn_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kTotal, st>>>(
       q, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared,
-      scale * kLog2e, g_fwd_safe_only.load(std::memory_order_relaxed), static_cast<__nv_bfloat16*>(o), lse);
+      scale * kLog2e, g_fwd_mode.load(std::memory_order_relaxed) == 1 ? 1 : 0, static_cast<__nv_bfloat16*>(o), lse);
   return launch_status();
 }
 
@@ -455,6 +504,8 @@ astro_status_t astro_chunk_attn_fwd(const astro_kvcache_t* cache, const void* q,
   const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q);
+  if (head_dim == 128 && g_fwd_mode.load(std::memory_order_relaxed) == 2)
+    return launch_fwd_pair(a, cache, have_ctx, q, k_chunk, v_chunk, segs, scale, o, lse, st);
   return head_dim == 128 ? launch_fwd<128>(a, qp, tkc, tvc, tkx, tvx, segs, scale, o, lse, st)
                          : launch_fwd<64>(a, qp, tkc, tvc, tkx, tvx, segs, scale, o, lse, st);
 }
@@ -632,8 +683,18 @@ astro_status_t astro_chunk_attn_bwd_static(const astro_kvcache_t* cache, const v
                                   dk_chunk, dv_chunk, stream);
 }
 
-astro_status_t astro_debug_forward_safe_only(int enable) {
-  g_fwd_safe_only.store(enable ? 1 : 0, std::memory_order_relaxed);
+astro_status_t astro_debug_forward_mode(int mode) {
+  if (mode < 0 || mode > 2) return ASTRO_ERR_SHAPE;
+  g_fwd_mode.store(mode, std::memory_order_relaxed);
+  return ASTRO_OK;
+}
+
+astro_status_t astro_debug_pair_flag(int* flag) {
+  if (!flag) return ASTRO_ERR_NULL;
+  if (cudaDeviceSynchronize() != cudaSuccess) return ASTRO_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(flag, g_pair_needs_safe, sizeof(int)) != cudaSuccess) return ASTRO_ERR_CUDA;
+  const int zero = 0;
+  if (cudaMemcpyToSymbol(g_pair_needs_safe, &zero, sizeof(zero)) != cudaSuccess) return ASTRO_ERR_CUDA;
   return ASTRO_OK;
 }
 

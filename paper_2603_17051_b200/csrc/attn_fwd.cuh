@@ -215,10 +215,10 @@ __device__ __forceinline__ float fwd_exp32(const uint32_t (&s)[32], int valid, f
 // Epilogue shared by both passes: row sum = sum of the groups' partial sums; 32-column slices of the output
 // row are dealt round-robin to the groups.  Returns false if a stored value was not finite.
 template <int D>
-__device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, const FwdBars& bar, int g, int r, uint32_t tmem_lane,
+__device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_full, int g, int r, uint32_t tmem_lane,
                                              float m_run, float l_run, bool in_range, __nv_bfloat16* dst,
                                              float* lse_dst) {
-  mbar_wait(bar.o_full, 0, u.abort_flag);
+  mbar_wait(o_full, 0, u.abort_flag);
   tc_fence_after_sync();
   float* ex = u.smax;  // free: the last exchange through it was consumed before the last P was published
   ex[g * kTile + r] = l_run;
@@ -311,7 +311,7 @@ __device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdB
     }
   }
   bool ok = (l_run < kFastSumLimit) && !(poly_max > kPolyArgLimit);   // false for inf and NaN too
-  ok = fwd_epilogue<D>(u, bar, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
+  ok = fwd_epilogue<D>(u, bar.o_full, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
   return ok;
 }
 
@@ -422,7 +422,7 @@ __device__ __forceinline__ void fwd_softmax_safe(const FwdUnit<D>& u, const FwdB
     tc_fence_before_sync();
     mbar_arrive(bar.p_full + g * kFwdSBufs + buf);
   }
-  fwd_epilogue<D>(u, bar, g, r, tmem_lane, m_run, l_run, in_range, dst, lse_dst);
+  fwd_epilogue<D>(u, bar.o_full, g, r, tmem_lane, m_run, l_run, in_range, dst, lse_dst);
 }
 
 template <int D>

@@ -188,3 +188,43 @@ def test_key_segments_cover_exactly_the_held_slots_in_every_ring_state():
         L.astro_kvcache_destroy(h)
     # no cache at all: only the chunk
     assert A.astro_kvcache_key_segments(None, 5) == [(0, 5, 1)]
+
+
+def test_two_threads_share_one_handle_for_validation_and_inspection():
+    """Attention calls take the cache as const: several host threads may issue them on one handle (the G candidates
+    of a group decoding against one shared prefix).  Here two threads hammer argument validation and the
+    key-segment inspection of one handle at the same time; every call must return the same answers as alone.
+    (What the calls do after validation needs a device and is covered by the GPU tests.)"""
+    import threading
+    L = A.lib()
+    d = A.KVCacheDesc(1, 2, 64, 16, 1, 4)
+    st, h = _raw_create(d)
+    assert st == 0
+    vp = C.c_void_p
+    results = [[], []]
+
+    def worker(slot):
+        n = C.c_int(); a, b, c = (C.c_int * 3)(), (C.c_int * 3)(), (C.c_int * 3)()
+        for _ in range(2000):
+            # misaligned q: rejected before anything is launched or any lazily built state is touched
+            r1 = L.astro_chunk_attn_fwd(h, vp(0x1008), vp(0x2000), vp(0x3000), 1, 2, 64, 8, 8, 0.1, vp(0x4000), None, None)
+            # a cache of other heads: shape error
+            r2 = L.astro_chunk_attn_fwd(h, vp(0x1000), vp(0x2000), vp(0x3000), 1, 3, 64, 8, 8, 0.1, vp(0x4000), None, None)
+            r3 = L.astro_kvcache_key_segments(h, 5, C.byref(n), a, b, c)
+            results[slot].append((r1, r2, r3, n.value, a[0], b[0], c[0]))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads: t.start()
+    for t in threads: t.join()
+    expect = (3, 2, 0, 1, 0, 5, 1)                       # ALIGN, SHAPE, OK and one chunk segment of 5 tokens
+    assert all(r == expect for res in results for r in res)
+    assert L.astro_kvcache_destroy(h) == 0
+
+
+def test_static_backward_rejects_misaligned_outputs_before_any_launch():
+    """A misaligned dK is an ASTRO_ERR_ALIGN up front (no device is needed to get the answer: nothing ran)."""
+    L = A.lib()
+    vp = C.c_void_p
+    st = L.astro_chunk_attn_bwd_static(None, vp(0x1000), vp(0x2000), vp(0x3000), vp(0x4000), vp(0x5000), vp(0x6000),
+                                       1, 2, 64, 8, 8, 0.1, vp(0x7000), vp(0x8008), vp(0x9000), None)
+    assert st == 3

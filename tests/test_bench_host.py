@@ -58,3 +58,29 @@ def test_reference_arm_prints_one_json_line():
     d = json.loads(out.stdout.strip().splitlines()[-1])
     assert d["impl"] == "reference" and d["unit"] == "TFLOP/s" and d["value"] > 0
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_plain_launch_with_gpus_2_starts_two_ranks():
+    """`bench.py --gpus 2` started without torchrun must start its two ranks itself; the dry run goes through the
+    rendezvous, the max-over-ranks reduction and the aggregate on CPU (gloo) and reports n_gpus = 2."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    env["MASTER_PORT"] = "29613"
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run", "--steps", "1",
+                          "--warmup", "0"], capture_output=True, text=True, env=env, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["dry_run"] is True
+    assert d["ms_per_step"] == 3.0                           # the slower rank's time
+    sys.path.insert(0, ROOT)
+    import bench
+    assert d["value"] == pytest.approx(bench.aggregate(bench.W.fwd_flops() + bench.W.bwd_flops(), 3.0, 2))
+
+
+def test_torchrun_command_uses_the_loopback_address():
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.torchrun_command(4, ["--gpus", "4"], port=29999)
+    assert "--master-addr" in cmd and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4" and cmd[-2:] == ["--gpus", "4"]

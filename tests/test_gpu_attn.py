@@ -37,9 +37,20 @@ def _fill(A, Bc, H, D, T, S, L, held, seed, churn=0):
 def safe_pass_only():
     """Every forward inside the test runs the kernel's safe pass (running row reference) instead of the fast one."""
     from paper_2603_17051_b200 import binding as A
-    A.astro_debug_forward_safe_only(True)
+    A.astro_debug_forward_mode(A.FWD_MODE_SAFE_ONLY)
     yield
-    A.astro_debug_forward_safe_only(False)
+    A.astro_debug_forward_mode(A.FWD_MODE_NORMAL)
+
+
+@pytest.fixture
+def pair_kernel():
+    """head_dim 128 forwards inside the test run the CTA-pair kernel; none of them may ask for the safe pass."""
+    from paper_2603_17051_b200 import binding as A
+    A.astro_debug_pair_flag()
+    A.astro_debug_forward_mode(A.FWD_MODE_PAIR)
+    yield
+    A.astro_debug_forward_mode(A.FWD_MODE_NORMAL)
+    assert A.astro_debug_pair_flag() == 0
 
 
 def _run_case(A, B, Bc, H, D, T, S, L, held, n_q, n_kc, seed, churn=0, evict_hole=0, scale=None, bwd=True,
@@ -126,6 +137,14 @@ def test_parity_cases(case):
     _run_case(A, **case)
 
 
+@pytest.mark.parametrize("case", [c for c in PARITY_CASES if c["D"] == 128])
+def test_parity_cases_pair_kernel(case, pair_kernel):
+    """The head_dim 128 cases through the CTA-pair kernel (two query tiles per K/V tile, cta_group::2 MMAs): odd and
+    even numbers of query tiles, ragged key ranges, holes, a shared prefix."""
+    from paper_2603_17051_b200 import binding as A
+    _run_case(A, bwd=False, **case)
+
+
 @pytest.mark.parametrize("case", PARITY_CASES)
 def test_parity_cases_safe_pass(case, safe_pass_only):
     """The same cases through the forward's safe pass (running row reference, O rescaled on the way)."""
@@ -166,10 +185,19 @@ def test_shared_prefix_equals_replicated_caches():
         assert torch.equal(a, b)
 
 
-def test_stale_nan_in_evicted_slots_does_not_leak():
+@pytest.mark.parametrize("mode", [0, 2])
+def test_stale_nan_in_evicted_slots_does_not_leak(mode):
     """Tile rows past a segment's end may hold anything (here NaN): results must not change."""
     import torch
     from paper_2603_17051_b200 import binding as A
+    A.astro_debug_forward_mode(mode)
+    try:
+        _stale_nan_case(A, torch)
+    finally:
+        A.astro_debug_forward_mode(0)
+
+
+def _stale_nan_case(A, torch):
     H, D, T, S, L = 2, 128, 50, 0, 4
     cache = A.astro_kvcache_create(1, H, D, T, S, L)
     cache.k_storage.view(torch.int16).fill_(0x7FC0 - 0x10000 if False else 0x7FC0)
@@ -347,11 +375,11 @@ def test_row_reference_follows_score_jumps_between_tiles(order, mode):
     the tile in its safe pass.  In the safe pass a row re-references itself whenever a tile's row sum leaves the
     safe range: several times per row (rising, steep), never after the first tile (falling), once (spike)."""
     from paper_2603_17051_b200 import binding as A
-    A.astro_debug_forward_safe_only(mode == "safe_pass")
+    A.astro_debug_forward_mode(A.FWD_MODE_SAFE_ONLY if mode == "safe_pass" else A.FWD_MODE_NORMAL)
     try:
         _score_jump_case(A, order)
     finally:
-        A.astro_debug_forward_safe_only(False)
+        A.astro_debug_forward_mode(A.FWD_MODE_NORMAL)
 
 
 def _score_jump_case(A, order):
@@ -455,3 +483,50 @@ def test_zero_scale_gives_uniform_attention():
     assert dq.float().abs().max() == 0 and dk.float().abs().max() == 0          # both carry the factor scale
     expect_dv = do.float().sum(dim=1, keepdim=True) / (4 * T + 140)
     assert (dv.float() - expect_dv).abs().max() < 2e-2
+
+
+def test_pair_kernel_reports_rows_that_need_the_safe_pass():
+    """The CTA-pair kernel keeps one reference per row; a key 100 nats above it overflows exp2 and must be reported."""
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, n_q, n_k = 1, 1, 128, 130, 128 * 2 + 9
+    qb = synth.f32_to_bf16_bits(np.ones((B, n_q, H, D), dtype=np.float32))
+    kf = np.zeros((B, n_k, H, D)); kf[:, 128 + 70] = 9.0
+    q, k, v = dev_bf16(qb), dev_bf16(synth.f32_to_bf16_bits(kf.astype(np.float32))), dev_bf16(synth.normal_bf16(4303, (B, n_k, H, D)))
+    A.astro_debug_pair_flag()
+    A.astro_debug_forward_mode(A.FWD_MODE_PAIR)
+    try:
+        A.astro_chunk_attn_fwd(None, q, k, v, 1.0 / np.sqrt(D))
+        A.astro_last_device_status()
+        assert A.astro_debug_pair_flag() == 1
+        A.astro_chunk_attn_fwd(None, q, k[:, :128].contiguous(), v[:, :128].contiguous(), 1.0 / np.sqrt(D))
+        assert A.astro_debug_pair_flag() == 0
+    finally:
+        A.astro_debug_forward_mode(A.FWD_MODE_NORMAL)
+
+
+@pytest.mark.parametrize("mode", [0, 2])
+def test_group_of_24_candidates_on_one_shared_prefix(mode):
+    """Clip-level group-wise sampling at full size: G = 24 candidate chunks (4680 queries each, 12 heads) decode
+    against ONE frozen prefix of 18 frames held once (cache_batch = 1); sampled rows of three candidates against
+    the oracle, in the normal kernel and in the CTA-pair kernel."""
+    from paper_2603_17051_b200 import binding as A
+    w = synth.LAYER_FWD
+    G, H, D, T, M = 24, w.heads, w.head_dim, w.tokens_per_frame, w.chunk_tokens
+    cache, model = _fill(A, 1, H, D, T, w.sink_frames, w.window_frames, w.held_frames, synth.tensor_seed(6, 0), churn=1)
+    bits = [synth.normal_bf16(synth.tensor_seed(6, 50 + i), (G, M, H, D)) for i in range(3)]
+    q, kc, vc = (dev_bf16(x) for x in bits)
+    A.astro_debug_pair_flag()
+    A.astro_debug_forward_mode(mode)
+    try:
+        o, lse = A.astro_chunk_attn_fwd(cache, q, kc, vc, w.scale)
+        A.astro_last_device_status()
+        assert A.astro_debug_pair_flag() == 0
+    finally:
+        A.astro_debug_forward_mode(0)
+    mk, mv = model.export()
+    rows = _sample_rows(M, 24, np.random.default_rng(6))
+    for (b, h) in ((0, 0), (11, 5), (23, 11)):
+        sl = lambda x: orc.bf16_bits_to_f64(x[b:b + 1, :, h:h + 1, :])
+        kx, vx = orc.bf16_bits_to_f64(mk[:, :, h:h + 1, :]), orc.bf16_bits_to_f64(mv[:, :, h:h + 1, :])
+        o_ref, lse_ref = orc.chunk_attn_fwd(sl(bits[0])[:, rows], kx, vx, sl(bits[1]), sl(bits[2]), w.scale)
+        check_fwd(o[b:b + 1, rows, h:h + 1], lse[b:b + 1, h:h + 1][:, :, rows], o_ref, lse_ref, tag="b%d h%d" % (b, h))
