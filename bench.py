@@ -532,13 +532,17 @@ def measure_rollout(A, dev, peaks, chunks=80, reading="A", steps=4):
     ms = s.elapsed_time(e)
     A.astro_last_device_status()
     frames = chunks * c
-    # append alone: 3 frames of K and V for all samples, read + written once (L2 flushed before each)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    t_app = []
-    for _ in range(12):
-        A.astro_kvcache_reset(cache); flush.zero_()
-        t_app.append(_event_ms(lambda: A.astro_kvcache_append(cache, kc, vc, c)))
-    app_ms = float(np.median(t_app[3:]))
+    # append alone: 3 frames of K and V for all samples, read + written once.  16 (evict, append) pairs back to back
+    # from four rotating source buffers (460 MB, larger than L2), so that neither the launch gap after a
+    # synchronise nor L2 hits on the source enter the figure
+    srcs = [(kc, vc)] + [(torch.empty_like(kc).copy_(kc), torch.empty_like(vc).copy_(vc)) for _ in range(3)]
+    def appends(n):
+        for i in range(n):
+            A.astro_kvcache_evict(cache, c)
+            A.astro_kvcache_append(cache, srcs[i & 3][0], srcs[i & 3][1], c)
+    appends(4)
+    app_ms = _event_ms(lambda: appends(16)) / 16
+    del srcs
     app_bytes = 2 * 2 * B * H * c * T * D * 2
     tf = flops / (ms * 1e-3) / 1e12
     regime = "burst" if ms < 1000.0 else "sustained"
@@ -604,6 +608,42 @@ def measure_score_sensitivity(A, dev, peaks, reps=10):
     return out
 
 
+def measure_pair_kernel(A, dev, peaks, reps=10):
+    """Forward on shapes of the workloads through the single-CTA kernel and through the CTA-pair kernel (two query
+    tiles per K/V tile, tcgen05 cta_group::2), one JSON-able row per shape."""
+    import torch
+    H, D, T = 12, 128, 1560
+    shapes = (("layer, B=1 (37 query tiles per head)", 1, 1, 18, 4680), ("rollout, B=4 per-sample caches, 12 held", 4, 4, 12, 4680),
+              ("group of 8 on one prefix", 8, 1, 18, 4680), ("group of 24 on one prefix", 24, 1, 18, 4680),
+              ("rl_update forward, B=2", 2, 2, 18, 4680), ("per-frame chunk, B=4, 20 held", 4, 4, 20, 1560),
+              ("B=8, 4608 queries (36 tiles per head)", 8, 8, 18, 4608))
+    rows = []
+    for name, B, Bc, held, M in shapes:
+        cache = A.astro_kvcache_create(Bc, H, D, T, 3, held, device=dev)
+        A.astro_kvcache_append(cache, _rnd(dev, 10, (Bc, held * T, H, D)), _rnd(dev, 11, (Bc, held * T, H, D)), held)
+        q, kc, vc = (_rnd(dev, i, (B, M, H, D)) for i in range(3))
+        o = torch.empty_like(q); lse = torch.empty((B, H, M), dtype=torch.float32, device=dev)
+        flops = 4.0 * B * H * M * (held * T + M) * D
+        row = {"shape": name, "batch": B, "cache_batch": Bc, "queries": M, "keys": held * T + M}
+        fwd = lambda: A.astro_chunk_attn_fwd(cache, q, kc, vc, 1.0 / float(np.sqrt(D)), o=o, lse=lse)
+        try:
+            for label, mode in (("single_cta", A.FWD_MODE_NORMAL), ("cta_pair", A.FWD_MODE_PAIR)):
+                A.astro_debug_forward_mode(mode)
+                for _ in range(3):
+                    fwd()
+                ms = _event_ms(fwd, reps)
+                row[label] = {"ms": ms, "tflops": flops / (ms * 1e-3) / 1e12}
+        finally:
+            A.astro_debug_forward_mode(A.FWD_MODE_NORMAL)
+        A.astro_last_device_status()
+        row["pair_needed_safe_pass"] = A.astro_debug_pair_flag()
+        row["pair_over_single_speed"] = row["single_cta"]["ms"] / row["cta_pair"]["ms"]
+        rows.append(row)
+        del cache, q, kc, vc, o, lse
+        torch.cuda.empty_cache()
+    return rows
+
+
 def measure_variants(A, dev, peaks, reps=20):
     """Window presets of Tab. S1 (S = 3; 21 or 15 frames attended in total, the chunk included) with 3-frame and
     with per-frame chunks: forward of one layer, batch 4."""
@@ -651,6 +691,10 @@ def run_extra(args):
     if args.workload == "variants":
         for row in measure_variants(A, dev, peaks):
             print(json.dumps(dict(workload="variants", **row)))
+        return 0
+    if args.workload == "pair":
+        for row in measure_pair_kernel(A, dev, peaks):
+            print(json.dumps(dict(workload="pair", **row)))
         return 0
     if args.workload == "sensitivity":
         print(json.dumps(measure_score_sensitivity(A, dev, peaks)))
@@ -759,7 +803,7 @@ def main():
     ap.add_argument("--no-legs", action="store_true", help="layer workload: skip the rollout / rl_update / variant sub-records")
     ap.add_argument("--rollout-chunks", type=int, default=16,
                     help="chunks of the rollout sub-record of the default line (the full workload has 80)")
-    ap.add_argument("--workload", choices=("layer", "rollout", "rl_update", "sweep", "group", "nft", "variants", "sensitivity"), default="layer",
+    ap.add_argument("--workload", choices=("layer", "rollout", "rl_update", "sweep", "group", "nft", "variants", "sensitivity", "pair"), default="layer",
                     help="layer (default): the contract line; the others print one JSON line per extra workload")
     ap.add_argument("--group", type=int, default=24, help="group workload: candidates G decoding against one prefix")
     ap.add_argument("--replicated", action="store_true",
