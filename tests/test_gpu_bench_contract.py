@@ -29,3 +29,13 @@ def test_default_bench_line_has_the_contract_keys():
     assert e["value"] > 0 and e["h2d_bytes_per_step"] == 4 * 4680 * 12 * 128 * 2
     assert e["d2h_bytes_per_step"] == 4 * 4680 * 12 * 128 * 2 + 12 * 4680 * 4
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+    # a 4-step region is far below a second: the burst figure is the denominator, the other fraction is beside it
+    assert "burst" in r["peak_source"] and r["frac"] == pytest.approx(r["frac_of_burst"])
+    assert r["traffic"] is None or r["traffic"] > 1e8
+    # both halves of the metric and their neighbours are timed in the same run
+    ro = d["rollout"]
+    assert ro["metric"] == "rollout_latent_frames_per_s" and ro["value"] > 0 and ro["chunks"] == 16
+    assert ro["append"]["bytes_moved"] == 2 * 2 * 4 * 12 * 3 * 1560 * 128 * 2 and 0 < ro["append"]["frac_of_hbm"] < 1.2
+    assert d["rl_update"]["fwd"]["tflops"] > 100 and d["rl_update"]["bwd"]["tflops"] > 100
+    assert [(v["attended_frames"], v["chunk_frames"]) for v in d["window_variants"]] == [(21, 3), (21, 1), (15, 3), (15, 1)]
+    assert 0.5 < d["score_sensitivity"]["slowdown_x8"] < 2.0
