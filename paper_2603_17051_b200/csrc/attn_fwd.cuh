@@ -8,8 +8,9 @@
 // 128 B/clk, the whole shared-memory bandwidth, and then competes with the TMA writes of the next tiles.
 // S of a whole key tile is one 128x128 MMA into one of two S buffers, issued two tiles ahead.  P is written
 // as bf16 pairs over the thread's own S columns and feeds P V from tensor memory.  K and V tiles travel
-// through 3-deep rings.  Part of the exponentials is evaluated by a polynomial on the FMA pipe, because
-// the special-function unit (16 exp2 per clock per SM) is as busy as the tensor core at head_dim 128.
+// through 3-deep rings.  A share of the exponentials can be evaluated by a polynomial on the FMA pipe instead of
+// the special-function unit (16 exp2 per clock per SM, as busy as the tensor core at head_dim 128); measured, the
+// polynomial's own FMA and integer work costs more than it saves, so the share is zero.
 //
 // The kernel makes up to two passes over the keys:
 //   fast pass  every row keeps ONE reference exponent, the maximum of its first key tile.  exp2(s - m) is
@@ -41,7 +42,9 @@ template <int D> struct FwdSmem {
   static constexpr int kTotal = kBars + 2 * kFwdBarSlots * 8 + 64 + 1024;  // + slack to align to 1024
 };
 
-constexpr int kPolyOf8 = 2;  // of every 8 pairs of exponentials, how many use the polynomial on the FMA pipe
+// Of every 8 pairs of exponentials, how many use the polynomial on the FMA pipe.  Layer shape, forward alone:
+// 0 -> 0.776 ms, 1 -> 0.781, 2 -> 0.802, 3 -> 0.828 in bursts; the same order under the power limit.
+constexpr int kPolyOf8 = 0;
 constexpr float kRowSumLimit = 1073741824.f;        // safe pass: a tile row sum beyond 2^30 re-references the row
 constexpr float kFastSumLimit = 1.2676506e30f;      // fast pass: a row sum beyond 2^100 sends the CTA to the safe pass
 constexpr float kPolyArgLimit = 126.f;              // largest exponent the polynomial exp2 may be handed
