@@ -102,20 +102,18 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
     // ------------------------------------------------------------------ TMA producer: this CTA's halves
     if (lane == 0) {
       KeyTileIter itk, itv;
-      int cache_seg_k = 0, cache_seg_v = 0;   // index of the cache range the iterator is in
       auto load_k = [&](int j) {
         const int st = j % kPairStages;
         const bool fc = itk.from_chunk(segs);
         mbar_wait_spin(bar.k_empty + st, ((j / kPairStages) & 1) ^ 1, abort_flag);
         if (rank == 0) mbar_arrive_expect_tx(bar.k_full + st, 2 * kPairHalfBytes);
         const uint32_t full = cluster_map(smem_u32(bar.k_full + st), 0);
-        const CUtensorMap* tm = fc ? &maps.kc : &maps.kx[itk.seg];
+        const CUtensorMap* tm = fc ? &maps.kc : &maps.kx[itk.seg];   // cache ranges come first in the list
         uint8_t* dst = sK + st * kPairHalfBytes;
         const int row = itk.row0(segs) + 64 * static_cast<int>(rank);
         tma_load_4d_pair(dst, tm, full, 0, row, h, fc ? b : bx);
         tma_load_4d_pair(dst + 64 * 128, tm, full, 64, row, h, fc ? b : bx);
         itk.next(segs);
-        (void)cache_seg_k;
       };
       auto load_v = [&](int j) {
         const int st = j % kPairStages;
@@ -127,7 +125,6 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
         tma_load_4d_pair(sV + st * kPairHalfBytes, tm, full, 64 * static_cast<int>(rank), itv.row0(segs), h,
                          fc ? b : bx);
         itv.next(segs);
-        (void)cache_seg_v;
       };
       for (int j = 0; j < kFwdSBufs && j < n_tiles; ++j) load_k(j);
       for (int j = 0; j < n_tiles; ++j) {
