@@ -451,6 +451,24 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   constexpr uint32_t kTmemCols = 512;
   constexpr int kMmaWarp = 4 * kFwdGroups, kTmaWarp = 4 * kFwdGroups + 1;
 
+  // Each softmax thread fetches its share of the Q row (64 elements: group g takes elements [64 g, 64 g + 64)) before
+  // anything else, so that the load's latency passes behind the barrier set-up and the tensor-memory allocation.
+  const int r = tid & 127;           // query row inside the tile = TMEM lane (softmax warps)
+  const int row = q0 + r;
+  const bool in_range = row < n_q;
+  const bool stages_q = warp < kMmaWarp && (warp >> 2) < D / 64;
+  uint32_t qr[32];
+  if (stages_q) {
+    const uint4* src = reinterpret_cast<const uint4*>(q + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + (warp >> 2) * 64);
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+      const uint4 t = in_range ? src[v] : make_uint4(0, 0, 0, 0);
+      qr[4 * v] = t.x; qr[4 * v + 1] = t.y; qr[4 * v + 2] = t.z; qr[4 * v + 3] = t.w;
+    }
+  }
+  if (warp == kTmaWarp && lane == 0) {
+    tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc); tma_prefetch_desc(&tm_kx); tma_prefetch_desc(&tm_vx);
+  }
   if (tid == 0) {
     bar_fast.init(128 * (D / 64), 128 * kFwdGroups);  // q_full: the threads that write Q into tensor memory
     bar_safe.init(1, 128);
@@ -478,9 +496,6 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   u.n_tiles = seg_tiles(segs);
   u.h = h; u.b = b; u.bx = cache_shared ? 0 : b;
 
-  const int r = tid & 127;           // query row inside the tile = TMEM lane (softmax warps)
-  const int row = q0 + r;
-  const bool in_range = row < n_q;
   __nv_bfloat16* dst = o + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D;
   float* lse_dst = lse ? lse + (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0) : nullptr;
 
@@ -490,20 +505,10 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   } else if (warp == kMmaWarp) {
     if (lane == 0 && !force_safe) fwd_issue<D, true>(u, bar_fast);
   } else {
-    // Q row -> tensor memory: 64-element halves of the row (32 packed columns each) are dealt to the groups
-    const int g = warp >> 2;
+    // Q row -> tensor memory (32 packed columns per 64 elements)
     const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-#pragma unroll
-    for (int hq = 0; hq < D / 64; ++hq) {
-      if (hq % kFwdGroups != g) continue;
-      uint32_t qr[32];
-      const uint4* src = reinterpret_cast<const uint4*>(q + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + hq * 64);
-#pragma unroll
-      for (int v = 0; v < 8; ++v) {
-        const uint4 t = in_range ? src[v] : make_uint4(0, 0, 0, 0);
-        qr[4 * v] = t.x; qr[4 * v + 1] = t.y; qr[4 * v + 2] = t.z; qr[4 * v + 3] = t.w;
-      }
-      tmem_st32(tmem_lane + kFwdColQ + hq * 32, qr);
+    if (stages_q) {
+      tmem_st32(tmem_lane + kFwdColQ + (warp >> 2) * 32, qr);
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(bar_fast.q_full);
