@@ -251,15 +251,15 @@ astro_status_t launch_fwd_pair(const AttnArgs& a, const astro_kvcache* cache, bo
 
 template <int D>
 astro_status_t launch_fwd(const AttnArgs& a, const __nv_bfloat16* q, const CUtensorMap& tkc, const CUtensorMap& tvc,
-                          const CUtensorMap& tkx, const CUtensorMap& tvx, const KeySegs& segs, float scale, void* o,
-                          float* lse, cudaStream_t st) {
+                          const CUtensorMap& tkx, const CUtensorMap (&tvx)[2], const KeySegs& segs, float scale,
+                          void* o, float* lse, cudaStream_t st) {
   static std::atomic<int> done[kMaxDevices];
   astro_status_t s = set_smem_once(chunk_attn_fwd_kernel<D>, FwdSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
   const int shared = (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
   dim3 grid((a.n_q + kTile - 1) / kTile, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
   chunk_attn_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kTotal, st>>>(
-      q, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared,
+      q, tkc, tvc, tkx, tvx[0], tvx[1], segs, a.n_q, a.heads, shared,
       scale * kLog2e, g_fwd_mode.load(std::memory_order_relaxed) == 1 ? 1 : 0, static_cast<__nv_bfloat16*>(o), lse);
   return launch_status();
 }
@@ -489,19 +489,25 @@ astro_status_t astro_chunk_attn_fwd(const astro_kvcache_t* cache, const void* q,
   s = check_arch();
   if (s != ASTRO_OK) return s;
   const bool have_ctx = cache && (cache->sink_held + cache->win_held) > 0;
-  CUtensorMap tkc, tvc, tkx, tvx;
+  CUtensorMap tkc, tvc, tkx, tvx[2];
   std::memset(&tkc, 0, sizeof(tkc)); std::memset(&tvc, 0, sizeof(tvc));
-  std::memset(&tkx, 0, sizeof(tkx)); std::memset(&tvx, 0, sizeof(tvx));
+  std::memset(&tkx, 0, sizeof(tkx)); std::memset(tvx, 0, sizeof(tvx));
   if (n_kc > 0) {
     if ((s = make_tmap_user(&tkc, k_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
     if ((s = make_tmap_user(&tvc, v_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
   }
+  const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
   if (have_ctx) {
     if ((s = cache_maps(cache)) != ASTRO_OK) return s;
     tkx = cache->tm_k;
-    tvx = cache->tm_v;
+    // V of each cache key range through a map that ends where the range ends: rows past it are zero-filled by
+    // TMA instead of carrying whatever an evicted or never written slot holds (0 * NaN would reach O)
+    for (int i = 0, ci = 0; i < segs.n; ++i) {
+      if (segs.from_chunk[i]) continue;
+      const long long end = static_cast<long long>(segs.start[i]) + segs.count[i];
+      if ((s = make_tmap_cache_range(&tvx[ci++], cache, cache->v, end, kTile)) != ASTRO_OK) return s;
+    }
   }
-  const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q);
   if (head_dim == 128 && g_fwd_mode.load(std::memory_order_relaxed) == 2)

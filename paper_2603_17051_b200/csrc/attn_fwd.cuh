@@ -16,9 +16,10 @@
 //   fast pass  every row keeps ONE reference exponent, the maximum of its first key tile.  exp2(s - m) is
 //              exact for any reference as long as nothing overflows (bf16 and fp32 share the exponent range,
 //              so later scores may exceed the reference by ~100 in log2 units), so O is never rescaled, the
-//              threads of a row never have to agree on anything after the first tile, and a thread hands
-//              its P to the MMA thread in two halves: P V of the first half runs while the second half is
-//              still being exponentiated.
+//              threads of a row never have to agree on anything after the first tile.  The MMA-issuing thread
+//              sets the pace, so everything a tile needs (the bytes of V(j) and K(j+2), every thread's P(j))
+//              arrives on ONE barrier and every burst of 16 MMAs (P V of tile j, S of tile j+2) is followed by
+//              ONE commit.
 //   safe pass  only if some row of the CTA saw a sum beyond 2^100, an infinity or a NaN in the fast pass: the
 //              whole tile is recomputed with a running reference that follows the row maximum (rescaling O
 //              and the row sums when a tile's row sum leaves the safe range).
@@ -73,7 +74,8 @@ struct FwdBars {
 
 // What every role of the CTA needs to know about its work unit.
 template <int D> struct FwdUnit {
-  const CUtensorMap *tm_kc, *tm_vc, *tm_kx, *tm_vx;
+  const CUtensorMap *tm_kc, *tm_vc, *tm_kx;
+  const CUtensorMap* tm_vx[2];   // one per cache key range, each ending where its range ends (rows past it read as 0)
   const KeySegs* segs;
   uint8_t *sK, *sV;
   float* smax;
@@ -104,7 +106,7 @@ __device__ __forceinline__ void fwd_produce(const FwdUnit<D>& u, const FwdBars& 
     const bool fc = itv.from_chunk(segs);
     mbar_wait_spin(bar.v_empty + st, ((j / kFwdVStages) & 1) ^ 1, u.abort_flag);
     mbar_arrive_expect_tx(bar.v_full + st, TileGeom<D>::kBytes);
-    tma_load_tile<D>(u.sV + st * TileGeom<D>::kBytes, fc ? u.tm_vc : u.tm_vx, bar.v_full + st, itv.row0(segs), u.h,
+    tma_load_tile<D>(u.sV + st * TileGeom<D>::kBytes, fc ? u.tm_vc : u.tm_vx[itv.seg], bar.v_full + st, itv.row0(segs), u.h,
                      fc ? u.b : u.bx);
     itv.next(segs);
   };
@@ -113,6 +115,84 @@ __device__ __forceinline__ void fwd_produce(const FwdUnit<D>& u, const FwdBars& 
     load_v(j);
     if (j + kFwdSBufs < u.n_tiles) load_k(j + kFwdSBufs);
   }
+}
+
+// ---------------------------------------------------------------------------------- fast pass: barriers
+// The MMA-issuing thread is the pace-maker of the kernel, so the fast pass gives it ONE wait and ONE commit per key
+// tile.  ready[j % 4] collects everything tile j needs: the bytes of V(j) and K(j+2) (the producer's arrive with the
+// byte count plus the TMA completions) and the arrival of every softmax thread that has stored its P(j).
+// sdone[t % 4] is committed behind S(t): S(t) is ready for the softmax threads, and -- MMAs complete in order --
+// the P V of tile t-2 is done too, so the producer may refill the K stage of tile t and the V stage of tile t-2.
+struct FwdFastBars {
+  uint64_t *q_full, *k01, *ready, *sdone, *o_full;
+  __device__ explicit FwdFastBars(uint64_t* b) : q_full(b), k01(b + 1), ready(b + 2), sdone(b + 6), o_full(b + 10) {}
+  __device__ void init(int q_count) const {
+    mbar_init(q_full, q_count);
+    mbar_init(k01, 1);
+    for (int i = 0; i < 4; ++i) { mbar_init(ready + i, 1 + 128 * kFwdGroups); mbar_init(sdone + i, 1); }
+    mbar_init(o_full, 1);
+  }
+};
+
+template <int D>
+__device__ __forceinline__ void fwd_produce_fast(const FwdUnit<D>& u, const FwdFastBars& bar) {
+  const KeySegs& segs = *u.segs;
+  KeyTileIter itk, itv;
+  auto load_k = [&](int j, uint64_t* full) {
+    const bool fc = itk.from_chunk(segs);
+    tma_load_tile<D>(u.sK + (j % kFwdKStages) * TileGeom<D>::kBytes, fc ? u.tm_kc : u.tm_kx, full, itk.row0(segs), u.h,
+                     fc ? u.b : u.bx);
+    itk.next(segs);
+  };
+  const int n01 = u.n_tiles < kFwdSBufs ? u.n_tiles : kFwdSBufs;
+  mbar_arrive_expect_tx(bar.k01, n01 * TileGeom<D>::kBytes);
+  for (int j = 0; j < n01; ++j) load_k(j, bar.k01);
+  for (int j = 0; j < u.n_tiles; ++j) {
+    // S(j-1) done: the K stage of tile j+2 (that of tile j-1) and the V stage of tile j (that of tile j-3) are free
+    if (j >= 1) mbar_wait_spin(bar.sdone + (j - 1) % 4, ((j - 1) / 4) & 1, u.abort_flag);
+    const bool more = j + kFwdSBufs < u.n_tiles;
+    uint64_t* full = bar.ready + j % 4;
+    mbar_arrive_expect_tx(full, (more ? 2 : 1) * TileGeom<D>::kBytes);
+    const bool fc = itv.from_chunk(segs);
+    tma_load_tile<D>(u.sV + (j % kFwdVStages) * TileGeom<D>::kBytes, fc ? u.tm_vc : u.tm_vx[itv.seg], full,
+                     itv.row0(segs), u.h, fc ? u.b : u.bx);
+    itv.next(segs);
+    if (more) load_k(j + kFwdSBufs, full);
+  }
+}
+
+template <int D>
+__device__ __forceinline__ void fwd_issue_fast(const FwdUnit<D>& u, const FwdFastBars& bar) {
+  const uint64_t k_desc0 = desc_kmajor(smem_u32(u.sK));
+  constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kTile, false, false);
+  constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);
+  const uint32_t tmem_base = u.tmem_base;
+  auto issue_s = [&](int j) {  // S(j) -> buffer j % 2; free because the PV of tile j-2 was issued before
+    const uint64_t k_desc = desc_step(k_desc0, (j % kFwdKStages) * TileGeom<D>::kBytes);
+#pragma unroll
+    for (int k = 0; k < D / 16; ++k)  // 16 elements of the head dimension = 8 packed Q columns
+      mma_ts(tmem_base + kFwdColS + (j % kFwdSBufs) * 128, tmem_base + kFwdColQ + k * 8,
+             desc_step(k_desc, (k >> 2) * TileGeom<D>::kBlockBytes + (k & 3) * 32), idesc_s, k > 0);
+    mma_commit(bar.sdone + j % 4);
+  };
+  mbar_wait_spin(bar.q_full, 0, u.abort_flag);
+  mbar_wait_spin(bar.k01, 0, u.abort_flag);
+  tc_fence_after_sync();
+  for (int j = 0; j < kFwdSBufs && j < u.n_tiles; ++j) issue_s(j);
+  for (int j = 0; j < u.n_tiles; ++j) {
+    const uint32_t pcol = tmem_base + kFwdColS + (j % kFwdSBufs) * 128;
+    const uint64_t v_desc = desc_mnmajor(smem_u32(u.sV + (j % kFwdVStages) * TileGeom<D>::kBytes), TileGeom<D>::kBlockBytes);
+    mbar_wait_spin(bar.ready + j % 4, (j / 4) & 1, u.abort_flag);
+    tc_fence_after_sync();
+#pragma unroll
+    for (int kb = 0; kb < kTile / 16; ++kb) {
+      // P of 16 keys = 8 packed columns; group g's pairs start at its own S columns
+      const uint32_t a = pcol + (kb * 16 / kFwdCols) * kFwdCols + (kb * 16 % kFwdCols) / 2;
+      mma_ts(tmem_base + kFwdColO, a, desc_step(v_desc, kb * 2048), idesc_pv, (j > 0 || kb > 0) ? 1u : 0u);
+    }
+    if (j + kFwdSBufs < u.n_tiles) issue_s(j + kFwdSBufs);
+  }
+  mma_commit(bar.o_full);
 }
 
 // ---------------------------------------------------------------------------------- MMA issuer (one thread)
@@ -262,7 +342,7 @@ __device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_fu
 // ---------------------------------------------------------------------------------- softmax, fast pass
 // Returns false if the row must be redone by the safe pass.
 template <int D>
-__device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdBars& bar, int warp, int r,
+__device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdFastBars& bar, int warp, int r,
                                                  float scale_log2, bool in_range, __nv_bfloat16* dst,
                                                  float* lse_dst) {
   const KeySegs& segs = *u.segs;
@@ -271,11 +351,9 @@ __device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdB
   float m_ref = 0.f, l_run = 0.f, poly_max = -INFINITY;
   int j = 0;
   for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
-    const int tile_valid = it.valid(segs);
-    const int valid = tile_valid - kFwdCols * g;  // valid keys of this group's share (may be <= 0)
-    const int buf = j % kFwdSBufs;
-    const uint32_t colS = kFwdColS + buf * 128 + g * kFwdCols;
-    mbar_wait(bar.s_full + buf, (j / kFwdSBufs) & 1, u.abort_flag);
+    const int valid = it.valid(segs) - kFwdCols * g;  // valid keys of this group's share (may be <= 0)
+    const uint32_t colS = kFwdColS + (j % kFwdSBufs) * 128 + g * kFwdCols;
+    mbar_wait(bar.sdone + j % 4, (j / 4) & 1, u.abort_flag);
     tc_fence_after_sync();
     uint32_t s[2][32];
     tmem_ld32(tmem_lane + colS, s[0]);
@@ -296,22 +374,17 @@ __device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdB
       m_ref = mx * scale_log2;
     }
     const float neg_m = -m_ref;
+    // V rows past a key range's end never hold stale data here: the cache ranges' tensor maps end with the range,
+    // the chunk's with the chunk, and TMA fills what lies beyond with zeros
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       uint32_t pk[16];
       l_run += fwd_exp32(s[half], valid - 32 * half, scale_log2, neg_m, pk, poly_max);
       tmem_st16(tmem_lane + colS + half * 16, pk);   // in place: this thread has read all of its S columns
-      if (half == 0 && g == 0 && tile_valid < kTile) {
-        // Rows past the segment's end may hold stale cache contents: P is 0 there, but 0 * NaN is NaN.
-        // Group 0 clears them before publishing its first half, which every PV MMA of the tile is issued after.
-        const int st = j % kFwdVStages;
-        mbar_wait(bar.v_full + st, (j / kFwdVStages) & 1, u.abort_flag);
-        zero_tile_rows_from<D>(u.sV + st * TileGeom<D>::kBytes, tile_valid, r);
-      }
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(bar.p_full + half * kFwdSBufs + buf);
     }
+    tmem_wait_st();
+    tc_fence_before_sync();
+    mbar_arrive(bar.ready + j % 4);
   }
   bool ok = (l_run < kFastSumLimit) && !(poly_max > kPolyArgLimit);   // false for inf and NaN too
   ok = fwd_epilogue<D>(u, bar.o_full, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
@@ -432,13 +505,15 @@ template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant__ CUtensorMap tm_kc,
                       const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kx,
-                      const __grid_constant__ CUtensorMap tm_vx, const __grid_constant__ KeySegs segs, const int n_q,
+                      const __grid_constant__ CUtensorMap tm_vx0, const __grid_constant__ CUtensorMap tm_vx1,
+                      const __grid_constant__ KeySegs segs, const int n_q,
                       const int heads, const int cache_shared, const float scale_log2, const int force_safe,
                       __nv_bfloat16* __restrict__ o, float* __restrict__ lse) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
   uint64_t* bar_mem = reinterpret_cast<uint64_t*>(smem + FwdSmem<D>::kBars);
-  const FwdBars bar_fast(bar_mem), bar_safe(bar_mem + kFwdBarSlots);
+  const FwdFastBars bar_fast(bar_mem);
+  const FwdBars bar_safe(bar_mem + kFwdBarSlots);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bar_mem + 2 * kFwdBarSlots);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   volatile int* redo_flag = reinterpret_cast<volatile int*>(tmem_holder + 2);
@@ -467,10 +542,10 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
     }
   }
   if (warp == kTmaWarp && lane == 0) {
-    tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc); tma_prefetch_desc(&tm_kx); tma_prefetch_desc(&tm_vx);
+    tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc); tma_prefetch_desc(&tm_kx); tma_prefetch_desc(&tm_vx0);
   }
   if (tid == 0) {
-    bar_fast.init(128 * (D / 64), 128 * kFwdGroups);  // q_full: the threads that write Q into tensor memory
+    bar_fast.init(128 * (D / 64));  // q_full: the threads that write Q into tensor memory
     bar_safe.init(1, 128);
     *abort_flag = 0;
     *redo_flag = force_safe;
@@ -486,7 +561,7 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   tc_fence_after_sync();
 
   FwdUnit<D> u;
-  u.tm_kc = &tm_kc; u.tm_vc = &tm_vc; u.tm_kx = &tm_kx; u.tm_vx = &tm_vx;
+  u.tm_kc = &tm_kc; u.tm_vc = &tm_vc; u.tm_kx = &tm_kx; u.tm_vx[0] = &tm_vx0; u.tm_vx[1] = &tm_vx1;
   u.segs = &segs;
   u.sK = smem + FwdSmem<D>::kK;
   u.sV = smem + FwdSmem<D>::kV;
@@ -501,9 +576,9 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
 
   // ---- fast pass
   if (warp == kTmaWarp) {
-    if (lane == 0 && !force_safe) fwd_produce<D>(u, bar_fast);
+    if (lane == 0 && !force_safe) fwd_produce_fast<D>(u, bar_fast);
   } else if (warp == kMmaWarp) {
-    if (lane == 0 && !force_safe) fwd_issue<D, true>(u, bar_fast);
+    if (lane == 0 && !force_safe) fwd_issue_fast<D>(u, bar_fast);
   } else {
     // Q row -> tensor memory (32 packed columns per 64 elements)
     const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
