@@ -276,7 +276,7 @@ astro_status_t launch_bwd_delta(const void* o, const void* d_o, int batch, int h
 
 template <int D>
 astro_status_t launch_bwd_dq(const AttnArgs& a, const __nv_bfloat16* q, const CUtensorMap& tdo, const CUtensorMap& tkc,
-                             const CUtensorMap& tvc, const CUtensorMap& tkx, const CUtensorMap& tvx,
+                             const CUtensorMap& tvc, const CUtensorMap (&tkx)[2], const CUtensorMap& tvx,
                              const KeySegs& segs, float scale, const float* lse, const float* delta, void* dq,
                              cudaStream_t st) {
   static std::atomic<int> done[kMaxDevices];
@@ -285,7 +285,7 @@ astro_status_t launch_bwd_dq(const AttnArgs& a, const __nv_bfloat16* q, const CU
   const int shared = (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
   dim3 grid_q((a.n_q + kTile - 1) / kTile, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
   chunk_attn_bwd_dq_kernel<D><<<grid_q, kDqThreads, DqSmem<D>::kTotal, st>>>(
-      q, tdo, tkc, tvc, tkx, tvx, segs, a.n_q, a.heads, shared, scale, lse, delta,
+      q, tdo, tkc, tvc, tkx[0], tkx[1], tvx, segs, a.n_q, a.heads, shared, scale, lse, delta,
       static_cast<__nv_bfloat16*>(dq));
   return launch_status();
 }
@@ -549,20 +549,26 @@ astro_status_t astro_chunk_attn_bwd_dq(const astro_kvcache_t* cache, const void*
   s = check_arch();
   if (s != ASTRO_OK) return s;
   const bool have_ctx = cache && (cache->sink_held + cache->win_held) > 0;
-  CUtensorMap tdo, tkc, tvc, tkx, tvx;
+  CUtensorMap tdo, tkc, tvc, tkx[2], tvx;
   std::memset(&tkc, 0, sizeof(tkc)); std::memset(&tvc, 0, sizeof(tvc));
-  std::memset(&tkx, 0, sizeof(tkx)); std::memset(&tvx, 0, sizeof(tvx));
+  std::memset(tkx, 0, sizeof(tkx)); std::memset(&tvx, 0, sizeof(tvx));
   if ((s = make_tmap_user(&tdo, d_o, head_dim, n_q, heads, batch)) != ASTRO_OK) return s;
   if (n_kc > 0) {
     if ((s = make_tmap_user(&tkc, k_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
     if ((s = make_tmap_user(&tvc, v_chunk, head_dim, n_kc, heads, batch)) != ASTRO_OK) return s;
   }
+  const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
   if (have_ctx) {
     if ((s = cache_maps(cache)) != ASTRO_OK) return s;
-    tkx = cache->tm_k;
     tvx = cache->tm_v;
+    // K of each cache key range through a map that ends where the range ends (rows past it are zeros: dS is 0
+    // there, but 0 * NaN from a stale slot would reach dQ)
+    for (int i = 0, ci = 0; i < segs.n; ++i) {
+      if (segs.from_chunk[i]) continue;
+      const long long end = static_cast<long long>(segs.start[i]) + segs.count[i];
+      if ((s = make_tmap_cache_range(&tkx[ci++], cache, cache->k, end, kTile)) != ASTRO_OK) return s;
+    }
   }
-  const KeySegs segs = build_segments(have_ctx ? cache : nullptr, n_kc);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q);
   return head_dim == 128 ? launch_bwd_dq<128>(a, qp, tdo, tkc, tvc, tkx, tvx, segs, scale, lse, delta, dq, st)

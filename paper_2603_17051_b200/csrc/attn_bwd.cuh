@@ -60,13 +60,23 @@ __global__ void __launch_bounds__(256) bwd_delta_kernel(const __nv_bfloat16* __r
 // groups still work on tile j.  dS = P o (dP - delta) goes to a bf16 buffer and dQ += dS K follows.  Q lives
 // in tensor memory (bf16 pairs, written once by the softmax threads) as the A operand of S, which takes a
 // quarter of the operand traffic off shared memory.
+// The MMA-issuing thread sets the pace of the kernel, so it gets two waits and two commits per key tile:
+//   rs[j % 4]  every thread has S(j) in registers AND the bytes of K(j+1) have landed -> S(j+1), commit s_full
+//   rb[j % 4]  every thread has stored dS(j) (so it has dP(j) in registers too) AND the bytes of V(j+1) have
+//              landed -> dP(j+1) and dQ(j) as one burst, commit b_done
+// b_done is committed once before the loop (behind dP(0)) and once per tile: commit number j+1 says dP(j) is
+// ready and dQ(j-1) is done, which frees the dS buffer, the K stage of tile j-1 and the V stage of tile j.  The
+// commits alternate between two barriers (commit k goes to b_done[k & 1]), because the producer may be asked
+// for commit k only after commit k+1 has happened, and a single barrier cannot be two phases ahead of a waiter.
+// Cache K goes through tensor maps that end where a key range ends, so rows past it are zeros, never stale data
+// (dS is 0 there, but 0 * NaN would reach dQ).
 //   TMEM columns: S [0,128)  dP [128,256)  dS [256,320)  Q [320,320+D/2)  dQ [384,384+D)
 constexpr int kDqKStages = 3, kDqVStages = 2;
 constexpr int kDqGroups = 2;                      // softmax groups: more warps per scheduler hide the
 constexpr int kDqCols = kTile / kDqGroups;         // exp2 latency behind the arithmetic of the other warps
 constexpr int kDqSoftmaxThreads = 128 * kDqGroups;
 constexpr int kDqThreads = kDqSoftmaxThreads + 64;
-constexpr int kDqPolyOf8 = 0;  // share of the exponentials on the FMA pipe: none pays here under the power limit
+constexpr int kDqPolyOf8 = 0;  // share of the exponentials on the FMA pipe: none pays (1.122 ms with 2/8 vs 1.086)
 
 template <int D> struct DqSmem {
   static constexpr int kdO = 0;
@@ -80,30 +90,24 @@ template <int D>
 __global__ void __launch_bounds__(kDqThreads, 1)
 chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant__ CUtensorMap tm_do,
                          const __grid_constant__ CUtensorMap tm_kc, const __grid_constant__ CUtensorMap tm_vc,
-                         const __grid_constant__ CUtensorMap tm_kx, const __grid_constant__ CUtensorMap tm_vx,
-                         const KeySegs segs, const int n_q, const int heads, const int cache_shared,
-                         const float scale, const float* __restrict__ lse, const float* __restrict__ delta,
-                         __nv_bfloat16* __restrict__ dq) {
+                         const __grid_constant__ CUtensorMap tm_kx0, const __grid_constant__ CUtensorMap tm_kx1,
+                         const __grid_constant__ CUtensorMap tm_vx, const __grid_constant__ KeySegs segs, const int n_q,
+                         const int heads, const int cache_shared, const float scale, const float* __restrict__ lse,
+                         const float* __restrict__ delta, __nv_bfloat16* __restrict__ dq) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = align_1024(smem_raw);
   uint8_t* sdO = smem + DqSmem<D>::kdO;
   uint8_t* sK = smem + DqSmem<D>::kK;
   uint8_t* sV = smem + DqSmem<D>::kV;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + DqSmem<D>::kBars);
-  uint64_t* q_full = bars;
-  uint64_t* k_full = bars + 1;                 // [kDqKStages]
-  uint64_t* k_empty = k_full + kDqKStages;
-  uint64_t* v_full = k_empty + kDqKStages;     // [kDqVStages]
-  uint64_t* v_empty = v_full + kDqVStages;
-  uint64_t* s_full = v_empty + kDqVStages;     // S(j) computed
-  uint64_t* dp_full = s_full + 1;              // dP(j) computed
-  uint64_t* s_free = dp_full + 1;              // 256 arrivals: every thread has S(j) in registers
-  uint64_t* dp_free = s_free + 1;              // 256 arrivals: every thread has dP(j) in registers
-  uint64_t* ds_full = dp_free + 1;             // every thread has written its part of dS(j)
-  uint64_t* dq_done = ds_full + 1;             // dQ(j) has consumed dS(j)
-  uint64_t* qt_full = dq_done + 1;             // Q is in tensor memory
-  uint64_t* dq_full = qt_full + 1;
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(dq_full + 1);
+  uint64_t* kv0_full = bars;                   // dO, K(0), V(0) have landed
+  uint64_t* qt_full = bars + 1;                // Q is in tensor memory
+  uint64_t* rs = bars + 2;                     // [4]
+  uint64_t* rb = bars + 6;                     // [4]
+  uint64_t* s_full = bars + 10;                // S(j) computed
+  uint64_t* b_done = bars + 11;                // [2], see above
+  uint64_t* dq_full = bars + 13;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 14);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -118,16 +122,12 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
   const int n_tiles = seg_tiles(segs);
 
   if (tid == 0) {
-    mbar_init(q_full, 1);
-    for (int i = 0; i < kDqKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
-    for (int i = 0; i < kDqVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
-    mbar_init(s_full, 1);
-    mbar_init(dp_full, 1);
-    mbar_init(s_free, kDqSoftmaxThreads);
-    mbar_init(dp_free, kDqSoftmaxThreads);
-    mbar_init(ds_full, kDqSoftmaxThreads);
-    mbar_init(dq_done, 1);
+    mbar_init(kv0_full, 1);
     mbar_init(qt_full, 128 * (D / 64));
+    for (int i = 0; i < 4; ++i) { mbar_init(rs + i, 1 + kDqSoftmaxThreads); mbar_init(rb + i, 1 + kDqSoftmaxThreads); }
+    mbar_init(s_full, 1);
+    mbar_init(b_done, 1);
+    mbar_init(b_done + 1, 1);
     mbar_init(dq_full, 1);
     *abort_flag = 0;
     fence_mbar_init();
@@ -144,20 +144,28 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
 
   if (warp == kTmaWarp) {
     if (lane == 0) {
-      mbar_arrive_expect_tx(q_full, TileGeom<D>::kBytes);
-      tma_load_tile<D>(sdO, &tm_do, q_full, q0, h, b);
-      int j = 0;
-      for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
-        const int sk = j % kDqKStages, sv = j % kDqVStages;
+      KeyTileIter it;
+      auto load_kv = [&](int t, uint64_t* k_bar, uint64_t* v_bar) {   // K(t), V(t) of the tile the iterator is on
         const bool fc = it.from_chunk(segs);
-        mbar_wait_spin(k_empty + sk, ((j / kDqKStages) & 1) ^ 1, abort_flag);
-        mbar_arrive_expect_tx(k_full + sk, TileGeom<D>::kBytes);
-        tma_load_tile<D>(sK + sk * TileGeom<D>::kBytes, fc ? &tm_kc : &tm_kx, k_full + sk, it.row0(segs), h,
+        const CUtensorMap* tk = fc ? &tm_kc : (it.seg == 0 ? &tm_kx0 : &tm_kx1);
+        tma_load_tile<D>(sK + (t % kDqKStages) * TileGeom<D>::kBytes, tk, k_bar, it.row0(segs), h, fc ? b : bx);
+        tma_load_tile<D>(sV + (t % kDqVStages) * TileGeom<D>::kBytes, fc ? &tm_vc : &tm_vx, v_bar, it.row0(segs), h,
                          fc ? b : bx);
-        mbar_wait_spin(v_empty + sv, ((j / kDqVStages) & 1) ^ 1, abort_flag);
-        mbar_arrive_expect_tx(v_full + sv, TileGeom<D>::kBytes);
-        tma_load_tile<D>(sV + sv * TileGeom<D>::kBytes, fc ? &tm_vc : &tm_vx, v_full + sv, it.row0(segs), h,
-                         fc ? b : bx);
+        it.next(segs);
+      };
+      mbar_arrive_expect_tx(kv0_full, 3 * TileGeom<D>::kBytes);
+      tma_load_tile<D>(sdO, &tm_do, kv0_full, q0, h, b);
+      load_kv(0, kv0_full, kv0_full);
+      for (int t = 1; t <= n_tiles; ++t) {
+        // commit t-1 of b_done: dQ(t-3) and dP(t-2) are done, the K stage and the V stage of tile t are free
+        if (t >= 2) mbar_wait_spin(b_done + ((t - 1) & 1), ((t - 2) >> 1) & 1, abort_flag);
+        if (t < n_tiles) {
+          mbar_arrive_expect_tx(rs + (t - 1) % 4, TileGeom<D>::kBytes);
+          mbar_arrive_expect_tx(rb + (t - 1) % 4, TileGeom<D>::kBytes);
+          load_kv(t, rs + (t - 1) % 4, rb + (t - 1) % 4);
+        } else {
+          mbar_arrive(rb + (t - 1) % 4);   // the last tile's burst waits for no bytes (its rs is never awaited)
+        }
       }
     }
   } else if (warp == kMmaWarp) {
@@ -165,10 +173,7 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
       constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kTile, false, false);
       const uint64_t k_desc0 = desc_kmajor(smem_u32(sK));
       auto issue_s = [&](int j) {
-        const int st = j % kDqKStages;
-        mbar_wait_spin(k_full + st, (j / kDqKStages) & 1, abort_flag);
-        tc_fence_after_sync();
-        const uint64_t k_desc = desc_step(k_desc0, st * TileGeom<D>::kBytes);
+        const uint64_t k_desc = desc_step(k_desc0, (j % kDqKStages) * TileGeom<D>::kBytes);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k)  // 16 elements of the head dimension = 8 packed Q columns
           mma_ts(tmem_base + kColS, tmem_base + kColQ + k * 8,
@@ -176,32 +181,26 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
         mma_commit(s_full);
       };
       auto issue_dp = [&](int j) {
-        const int st = j % kDqVStages;
-        mbar_wait_spin(v_full + st, (j / kDqVStages) & 1, abort_flag);
-        tc_fence_after_sync();
-        mma_abT<D>(tmem_base + kColdP, smem_u32(sdO), smem_u32(sV + st * TileGeom<D>::kBytes));
-        mma_commit(v_empty + st);
-        mma_commit(dp_full);
+        mma_abT<D>(tmem_base + kColdP, smem_u32(sdO), smem_u32(sV + (j % kDqVStages) * TileGeom<D>::kBytes));
       };
       mbar_wait_spin(qt_full, 0, abort_flag);
-      mbar_wait_spin(q_full, 0, abort_flag);
+      mbar_wait_spin(kv0_full, 0, abort_flag);
       tc_fence_after_sync();
       issue_s(0);
       issue_dp(0);
+      mma_commit(b_done + 1);                       // commit 1
       for (int j = 0; j < n_tiles; ++j) {
-        if (j + 1 < n_tiles) {
-          mbar_wait_spin(s_free, j & 1, abort_flag);   // S(j) is in registers everywhere
+        const bool more = j + 1 < n_tiles;
+        if (more) {
+          mbar_wait_spin(rs + j % 4, (j / 4) & 1, abort_flag);
+          tc_fence_after_sync();
           issue_s(j + 1);
-          mbar_wait_spin(dp_free, j & 1, abort_flag);  // dP(j) is in registers everywhere
-          issue_dp(j + 1);
         }
-        const int st = j % kDqKStages;
-        const uint32_t kt = smem_u32(sK + st * TileGeom<D>::kBytes);
-        mbar_wait_spin(ds_full, j & 1, abort_flag);
+        mbar_wait_spin(rb + j % 4, (j / 4) & 1, abort_flag);
         tc_fence_after_sync();
-        mma_pb<D, kTile>(tmem_base + kColdQ, tmem_base + kColdS, kt, j > 0);
-        mma_commit(k_empty + st);
-        mma_commit(dq_done);
+        if (more) issue_dp(j + 1);
+        mma_pb<D, kTile>(tmem_base + kColdQ, tmem_base + kColdS, smem_u32(sK + (j % kDqKStages) * TileGeom<D>::kBytes), j > 0);
+        mma_commit(b_done + (j & 1));                 // commit j + 2
       }
       mma_commit(dq_full);
     }
@@ -232,8 +231,7 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
     }
     int j = 0;
     for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
-      const int tile_valid = it.valid(segs);
-      const int valid = tile_valid - kDqCols * g;  // valid keys of this group's share (may be <= 0)
+      const int valid = it.valid(segs) - kDqCols * g;  // valid keys of this group's share (may be <= 0)
       mbar_wait(s_full, j & 1, abort_flag);
       tc_fence_after_sync();
       constexpr int NL = kDqCols / 32;
@@ -242,7 +240,7 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
       for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + kColS + g * kDqCols + c2 * 32, s[c2]);
       tmem_wait_ld();
       tc_fence_before_sync();
-      mbar_arrive(s_free);
+      mbar_arrive(rs + j % 4);
       // P = exp2(s * scale * log2e - LSE * log2e), kept as packed fp32 pairs
       uint64_t p2[NL][16];
 #pragma unroll
@@ -261,14 +259,13 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
           }
           p2[c2][c >> 1] = f32x2(p0, p1);
         }
-      mbar_wait(dp_full, j & 1, abort_flag);
+      // commit j+1 of b_done: dP(j) is there, and dQ(j-1) has consumed the one dS buffer
+      mbar_wait(b_done + ((j + 1) & 1), (j >> 1) & 1, abort_flag);
       tc_fence_after_sync();
       uint32_t dp[NL][32], ds[NL][16];
 #pragma unroll
       for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + kColdP + g * kDqCols + c2 * 32, dp[c2]);
       tmem_wait_ld();
-      tc_fence_before_sync();
-      mbar_arrive(dp_free);
 #pragma unroll
       for (int c2 = 0; c2 < NL; ++c2)
 #pragma unroll
@@ -277,25 +274,18 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
                                    add2(f32x2(__uint_as_float(dp[c2][c]), __uint_as_float(dp[c2][c + 1])), nd2));
           float d0, d1;
           f32x2_split(d2, d0, d1);
-          if (valid < kDqCols) {  // stale keys past the segment's end: S and dP hold anything, dS must be 0
+          if (valid < kDqCols) {  // keys past the segment's end: S and dP hold anything, dS must be 0
             if (c2 * 32 + c >= valid) d0 = 0.f;
             if (c2 * 32 + c + 1 >= valid) d1 = 0.f;
           }
           ds[c2][c >> 1] = pack_bf16(d0, d1);
         }
-      if (j > 0) {  // the one dS buffer is free once dQ(j-1) has consumed it (almost always long since)
-        mbar_wait(dq_done, (j - 1) & 1, abort_flag);
-        tc_fence_after_sync();
-      }
 #pragma unroll
       for (int c2 = 0; c2 < NL; ++c2)
         tmem_st16(tmem_lane + kColdS + g * (kDqCols / 2) + c2 * 16, ds[c2]);
-      // Key rows past the segment's end may hold stale cache contents: dS is 0 there, but 0 * NaN is NaN.
-      if (g == 0 && tile_valid < kTile)
-        zero_tile_rows_from<D>(sK + (j % kDqKStages) * TileGeom<D>::kBytes, tile_valid, r);
       tmem_wait_st();
       tc_fence_before_sync();
-      mbar_arrive(ds_full);
+      mbar_arrive(rb + j % 4);   // dS(j) stored; dP(j) was read before it, so its buffer is free as well
     }
     // ---- epilogue: groups 0 and 1 write columns [g D/2, (g+1) D/2) of dQ
     mbar_wait(dq_full, 0, abort_flag);
