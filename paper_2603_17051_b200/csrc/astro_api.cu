@@ -243,7 +243,7 @@ astro_status_t launch_fwd_pair(const AttnArgs& a, const astro_kvcache* cache, bo
   const int shared = (cache && cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
   const int tiles = (a.n_q + kTile - 1) / kTile;
   dim3 grid((tiles + 1) / 2 * 2, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
-  chunk_attn_fwd_pair_kernel<<<grid, kFwdThreads, PairSmem::kTotal, st>>>(
+  chunk_attn_fwd_pair_kernel<<<grid, kPairThreads, PairSmem::kTotal, st>>>(
       static_cast<const __nv_bfloat16*>(q), maps, segs, a.n_q, a.heads, shared, scale * kLog2e,
       static_cast<__nv_bfloat16*>(o), lse, flag);
   return launch_status();

@@ -1,8 +1,9 @@
 // Forward of chunk attention over the rolling cache: O and LSE for one 128-query tile per CTA.
 //
 // Warp-specialised, one CTA per SM:
-//   two softmax groups of 4 warps: group g owns keys [64 g, 64 g + 64) of every key tile, one query row
-//   per thread; then one warp whose first thread issues every tcgen05 MMA, one for TMA loads
+//   four softmax groups of 4 warps: group g owns keys [32 g, 32 g + 32) of every key tile, one query row
+//   per thread (four warps per scheduler: while one waits for tensor memory or a barrier the others keep the
+//   special-function unit busy); then one warp whose first thread issues every tcgen05 MMA, one for TMA loads
 // Q lives in tensor memory (bf16 pairs, written once by the softmax threads) and is the A operand of
 // S = Q K^T, so shared memory only carries K and V: an MMA with both operands in shared memory reads
 // 128 B/clk, the whole shared-memory bandwidth, and then competes with the TMA writes of the next tiles.
@@ -30,10 +31,10 @@
 namespace astro {
 
 constexpr int kFwdKStages = 3, kFwdVStages = 3, kFwdSBufs = 2;
-constexpr int kFwdGroups = 2;                    // more warps per scheduler hide the exp2 latency
+constexpr int kFwdGroups = 4;                    // layer shape, forward alone: 2 groups 0.741 ms, 4 groups 0.713 ms
 constexpr int kFwdCols = kTile / kFwdGroups;     // keys per group and tile
 constexpr int kFwdThreads = 128 * kFwdGroups + 64;
-constexpr int kFwdBarSlots = 24;                 // mbarriers of one pass
+constexpr int kFwdBarSlots = 32;                 // mbarriers of one pass
 
 template <int D> struct FwdSmem {
   static constexpr int kK = 0;
@@ -50,22 +51,22 @@ constexpr float kRowSumLimit = 1073741824.f;        // safe pass: a tile row sum
 constexpr float kFastSumLimit = 1.2676506e30f;      // fast pass: a row sum beyond 2^100 sends the CTA to the safe pass
 constexpr float kPolyArgLimit = 126.f;              // largest exponent the polynomial exp2 may be handed
 
-// The mbarriers of one pass.  The two passes use separate sets, so a late arrival of the first pass can
+// The mbarriers of the safe pass.  The two passes use separate sets, so a late arrival of the first pass can
 // never land in a phase of the second.
 struct FwdBars {
   uint64_t *q_full, *k_full, *k_empty, *v_full, *v_empty, *s_full, *p_full, *pv_done, *o_full;
   __device__ explicit FwdBars(uint64_t* b)
       : q_full(b), k_full(b + 1), k_empty(k_full + kFwdKStages), v_full(k_empty + kFwdKStages),
         v_empty(v_full + kFwdVStages), s_full(v_empty + kFwdVStages), p_full(s_full + kFwdSBufs),
-        pv_done(p_full + 2 * kFwdSBufs), o_full(pv_done + 2) {}
-  // p_full: safe pass [group][S buffer], 128 arrivals each (the groups may run up to two tiles ahead of the
-  // MMA thread, so the barriers rotate with the S buffers); fast pass [half][S buffer], 256 arrivals each.
+        pv_done(p_full + kFwdGroups * kFwdSBufs), o_full(pv_done + 2) {}
+  // p_full [group][S buffer], 128 arrivals each: the groups may run up to two tiles ahead of the MMA thread, so
+  // the barriers rotate with the S buffers.
   __device__ void init(int q_count, int p_count) const {
     mbar_init(q_full, q_count);
     for (int i = 0; i < kFwdKStages; ++i) { mbar_init(k_full + i, 1); mbar_init(k_empty + i, 1); }
     for (int i = 0; i < kFwdVStages; ++i) { mbar_init(v_full + i, 1); mbar_init(v_empty + i, 1); }
     for (int i = 0; i < kFwdSBufs; ++i) mbar_init(s_full + i, 1);
-    for (int i = 0; i < 2 * kFwdSBufs; ++i) mbar_init(p_full + i, p_count);
+    for (int i = 0; i < kFwdGroups * kFwdSBufs; ++i) mbar_init(p_full + i, p_count);
     mbar_init(pv_done, 1);
     mbar_init(pv_done + 1, 1);
     mbar_init(o_full, 1);
@@ -200,9 +201,9 @@ __device__ __forceinline__ void fwd_issue_fast(const FwdUnit<D>& u, const FwdFas
 // executes, the queue behind it is short), so every clock this thread spends on anything else is an idle clock of
 // the pipe.  Per key tile it therefore first makes sure of everything the tile needs (V(j), K(j+2), P(j)), then
 // issues P V of tile j and S of tile j+2 as one uninterrupted burst of 16 MMAs, then commits.
-// kFast: P of a tile arrives in two halves per group (p_full[half][buffer]).  Otherwise P arrives per group
-// (p_full[group][buffer]); any of the groups may have rescaled its part of O before it published.
-template <int D, bool kFast>
+// Safe pass: P arrives per group (p_full[group][buffer]); any of the groups may have rescaled its part of O before
+// it published, so all of them are awaited first.
+template <int D>
 __device__ __forceinline__ void fwd_issue(const FwdUnit<D>& u, const FwdBars& bar) {
   const uint64_t k_desc0 = desc_kmajor(smem_u32(u.sK));
   constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kTile, false, false);
@@ -222,7 +223,6 @@ __device__ __forceinline__ void fwd_issue(const FwdUnit<D>& u, const FwdBars& ba
     mma_commit(bar.k_empty + j % kFwdKStages);
     mma_commit(bar.s_full + j % kFwdSBufs);
   };
-  if (kFast) mbar_wait_spin(bar.q_full, 0, u.abort_flag);
   for (int j = 0; j < kFwdSBufs && j < u.n_tiles; ++j) {
     wait_k(j);
     tc_fence_after_sync();
@@ -237,8 +237,8 @@ __device__ __forceinline__ void fwd_issue(const FwdUnit<D>& u, const FwdBars& ba
     mbar_wait_spin(bar.v_full + st, (j / kFwdVStages) & 1, u.abort_flag);
     if (more) wait_k(j + kFwdSBufs);
 #pragma unroll
-    for (int i = 0; i < 2; ++i)   // halves (fast pass) or groups (safe pass)
-      mbar_wait_spin(bar.p_full + i * kFwdSBufs + buf, (j / kFwdSBufs) & 1, u.abort_flag);
+    for (int g = 0; g < kFwdGroups; ++g)
+      mbar_wait_spin(bar.p_full + g * kFwdSBufs + buf, (j / kFwdSBufs) & 1, u.abort_flag);
     tc_fence_after_sync();
 #pragma unroll
     for (int kb = 0; kb < kTile / 16; ++kb) {
@@ -247,7 +247,7 @@ __device__ __forceinline__ void fwd_issue(const FwdUnit<D>& u, const FwdBars& ba
       mma_ts(tmem_base + kFwdColO, a, desc_step(v_desc, kb * 2048), idesc_pv, (j > 0 || kb > 0) ? 1u : 0u);
     }
     if (more) issue_s(j + kFwdSBufs);
-    if (!kFast) mma_commit(bar.pv_done + (j & 1));   // tracks the S MMAs too: they are long done when O is needed
+    mma_commit(bar.pv_done + (j & 1));   // tracks the S MMAs too: they are long done when O is needed
     mma_commit(bar.v_empty + st);
     if (more) commit_s(j + kFwdSBufs);
   }
@@ -297,7 +297,7 @@ __device__ __forceinline__ float fwd_exp32(const uint32_t (&s)[32], int valid, f
 
 // Epilogue shared by both passes: row sum = sum of the groups' partial sums; 32-column slices of the output
 // row are dealt round-robin to the groups.  Returns false if a stored value was not finite.
-template <int D>
+template <int D, int G = kFwdGroups>
 __device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_full, int g, int r, uint32_t tmem_lane,
                                              float m_run, float l_run, bool in_range, __nv_bfloat16* dst,
                                              float* lse_dst) {
@@ -305,15 +305,15 @@ __device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_fu
   tc_fence_after_sync();
   float* ex = u.smax;  // free: the last exchange through it was consumed before the last P was published
   ex[g * kTile + r] = l_run;
-  named_barrier_sync(5, 128 * kFwdGroups);
+  named_barrier_sync(5, 128 * G);
   float l = 0.f;
 #pragma unroll
-  for (int og = 0; og < kFwdGroups; ++og) l += ex[og * kTile + r];
+  for (int og = 0; og < G; ++og) l += ex[og * kTile + r];
   const float inv_l = 1.f / l;
   uint32_t worst = 0;
 #pragma unroll
   for (int c4 = 0; c4 < D / 32; ++c4) {
-    if (c4 % kFwdGroups != g) continue;
+    if (c4 % G != g) continue;
     uint32_t acc[32];
     tmem_ld32(tmem_lane + kFwdColO + c4 * 32, acc);
     tmem_wait_ld();
@@ -355,32 +355,34 @@ __device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdF
     const uint32_t colS = kFwdColS + (j % kFwdSBufs) * 128 + g * kFwdCols;
     mbar_wait(bar.sdone + j % 4, (j / 4) & 1, u.abort_flag);
     tc_fence_after_sync();
-    uint32_t s[2][32];
-    tmem_ld32(tmem_lane + colS, s[0]);
-    tmem_ld32(tmem_lane + colS + 32, s[1]);
+    constexpr int NL = kFwdCols / 32;  // 32-column TMEM loads per thread and tile
+    uint32_t s[NL][32];
+#pragma unroll
+    for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);
     tmem_wait_ld();
     if (j == 0) {
-      // the row's one reference: the maximum of the first tile, agreed between the two threads of the row
+      // the row's one reference: the maximum of the first tile, agreed between the threads of the row
       float mx = -INFINITY;
 #pragma unroll
-      for (int c2 = 0; c2 < 2; ++c2)
+      for (int c2 = 0; c2 < NL; ++c2)
 #pragma unroll
         for (int c = 0; c < 32; ++c)
           if (c2 * 32 + c < valid) mx = fmaxf(mx, __uint_as_float(s[c2][c]));
       float* mslot = u.smax + 2 * kFwdGroups * kTile;
       mslot[g * kTile + r] = mx;
       named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
-      mx = fmaxf(mx, mslot[(g ^ 1) * kTile + r]);   // finite unless the inputs are not: >= 1 valid key
+#pragma unroll
+      for (int og = 0; og < kFwdGroups; ++og) mx = fmaxf(mx, mslot[og * kTile + r]);  // finite: >= 1 valid key
       m_ref = mx * scale_log2;
     }
     const float neg_m = -m_ref;
     // V rows past a key range's end never hold stale data here: the cache ranges' tensor maps end with the range,
     // the chunk's with the chunk, and TMA fills what lies beyond with zeros
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
+    for (int c2 = 0; c2 < NL; ++c2) {
       uint32_t pk[16];
-      l_run += fwd_exp32(s[half], valid - 32 * half, scale_log2, neg_m, pk, poly_max);
-      tmem_st16(tmem_lane + colS + half * 16, pk);   // in place: this thread has read all of its S columns
+      l_run += fwd_exp32(s[c2], valid - 32 * c2, scale_log2, neg_m, pk, poly_max);
+      tmem_st16(tmem_lane + colS + c2 * 16, pk);   // in place: this thread has read all of its S columns
     }
     tmem_wait_st();
     tc_fence_before_sync();
@@ -600,7 +602,7 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
     if (warp == kTmaWarp) {
       if (lane == 0) fwd_produce<D>(u, bar_safe);
     } else if (warp == kMmaWarp) {
-      if (lane == 0) fwd_issue<D, false>(u, bar_safe);
+      if (lane == 0) fwd_issue<D>(u, bar_safe);
     } else {
       fwd_softmax_safe<D>(u, bar_safe, warp, r, scale_log2, in_range, dst, lse_dst);
     }

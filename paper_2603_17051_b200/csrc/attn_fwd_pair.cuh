@@ -19,13 +19,16 @@
 namespace astro {
 
 constexpr int kPairStages = 4;
+constexpr int kPairGroups = 2;                       // softmax groups per CTA: 64 keys of a tile each
+constexpr int kPairCols = kTile / kPairGroups;
+constexpr int kPairThreads = 128 * kPairGroups + 64;
 constexpr int kPairHalfBytes = 64 * 128 * 2;   // 64 keys x 128 d of K (2 blocks of 64 rows), or 128 keys x 64 d of V
 
 struct PairSmem {
   static constexpr int kK = 0;
   static constexpr int kV = kK + kPairStages * kPairHalfBytes;
   static constexpr int kMax = kV + kPairStages * kPairHalfBytes;   // float [3][groups][128]
-  static constexpr int kBars = kMax + 3 * kFwdGroups * kTile * 4;
+  static constexpr int kBars = kMax + 3 * kPairGroups * kTile * 4;
   static constexpr int kTotal = kBars + 32 * 8 + 64 + 1024;
 };
 
@@ -44,11 +47,11 @@ struct PairBars {
         v_empty(k_empty + kPairStages), s_full(v_empty + kPairStages), p_full(s_full + kFwdSBufs),
         o_full(p_full + kFwdSBufs) {}
   __device__ void init() const {
-    mbar_init(q_full, 2 * 128 * kFwdGroups);
+    mbar_init(q_full, 2 * 128 * kPairGroups);
     for (int i = 0; i < kPairStages; ++i) {
       mbar_init(k_full + i, 1); mbar_init(v_full + i, 1); mbar_init(k_empty + i, 1); mbar_init(v_empty + i, 1);
     }
-    for (int i = 0; i < kFwdSBufs; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 2 * 4 * kFwdGroups); }
+    for (int i = 0; i < kFwdSBufs; ++i) { mbar_init(s_full + i, 1); mbar_init(p_full + i, 2 * 4 * kPairGroups); }
     mbar_init(o_full, 1);
   }
 };
@@ -58,7 +61,7 @@ struct PairMaps {
   CUtensorMap kx[2], vx[2];  // the cache key ranges, each map ending where its range ends
 };
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant__ PairMaps maps,
                            const __grid_constant__ KeySegs segs, const int n_q, const int heads, const int cache_shared,
                            const float scale_log2, __nv_bfloat16* __restrict__ o, float* __restrict__ lse,
@@ -79,7 +82,7 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
   const int h = cache_shared ? blockIdx.z : blockIdx.y, b = cache_shared ? blockIdx.y : blockIdx.z;
   const int bx = cache_shared ? 0 : b;
   constexpr uint32_t kTmemCols = 512;
-  constexpr int kMmaWarp = 4 * kFwdGroups, kTmaWarp = 4 * kFwdGroups + 1;
+  constexpr int kMmaWarp = 4 * kPairGroups, kTmaWarp = 4 * kPairGroups + 1;
   const int n_tiles = seg_tiles(segs);
 
   if (tid == 0) {
@@ -164,7 +167,7 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
         tc_fence_after_sync();
 #pragma unroll
         for (int kb = 0; kb < kTile / 16; ++kb) {
-          const uint32_t a = pcol + (kb * 16 / kFwdCols) * kFwdCols + (kb * 16 % kFwdCols) / 2;
+          const uint32_t a = pcol + (kb * 16 / kPairCols) * kPairCols + (kb * 16 % kPairCols) / 2;
           mma_ts_pair(tmem_base + kFwdColO, a, desc_step(v_desc, kb * 2048), idesc_pv, (j > 0 || kb > 0) ? 1u : 0u);
         }
         if (more) issue_s(jn);
@@ -201,9 +204,9 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
     float m_ref = 0.f, l_run = 0.f, poly_max = -INFINITY;
     int j = 0;
     for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
-      const int valid = it.valid(segs) - kFwdCols * g;
+      const int valid = it.valid(segs) - kPairCols * g;
       const int buf = j % kFwdSBufs;
-      const uint32_t colS = kFwdColS + buf * 128 + g * kFwdCols;
+      const uint32_t colS = kFwdColS + buf * 128 + g * kPairCols;
       mbar_wait(bar.s_full + buf, (j / kFwdSBufs) & 1, abort_flag);
       tc_fence_after_sync();
       uint32_t s[2][32];
@@ -217,9 +220,9 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
 #pragma unroll
           for (int c = 0; c < 32; ++c)
             if (c2 * 32 + c < valid) mx = fmaxf(mx, __uint_as_float(s[c2][c]));
-        float* mslot = smax + 2 * kFwdGroups * kTile;
+        float* mslot = smax + 2 * kPairGroups * kTile;
         mslot[g * kTile + r] = mx;
-        named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
+        named_barrier_sync(1 + (warp & 3), 32 * kPairGroups);
         mx = fmaxf(mx, mslot[(g ^ 1) * kTile + r]);
         m_ref = mx * scale_log2;
       }
@@ -241,7 +244,7 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
     u.abort_flag = abort_flag;
     __nv_bfloat16* dst = o + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D;
     float* lse_dst = lse ? lse + (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0) : nullptr;
-    ok = fwd_epilogue<D>(u, bar.o_full, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
+    ok = fwd_epilogue<D, kPairGroups>(u, bar.o_full, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
     if (!ok) *needs_safe = 1;
   }
 
