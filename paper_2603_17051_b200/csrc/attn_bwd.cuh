@@ -266,20 +266,31 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
 #pragma unroll
       for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + kColdP + g * kDqCols + c2 * 32, dp[c2]);
       tmem_wait_ld();
+      if (valid >= kDqCols) {   // the usual tile: no key to mask, nothing but the algebra in the loop
 #pragma unroll
-      for (int c2 = 0; c2 < NL; ++c2)
+        for (int c2 = 0; c2 < NL; ++c2)
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const uint64_t d2 = mul2(p2[c2][c >> 1],
-                                   add2(f32x2(__uint_as_float(dp[c2][c]), __uint_as_float(dp[c2][c + 1])), nd2));
-          float d0, d1;
-          f32x2_split(d2, d0, d1);
-          if (valid < kDqCols) {  // keys past the segment's end: S and dP hold anything, dS must be 0
+          for (int c = 0; c < 32; c += 2) {
+            const uint64_t d2 = mul2(p2[c2][c >> 1],
+                                     add2(f32x2(__uint_as_float(dp[c2][c]), __uint_as_float(dp[c2][c + 1])), nd2));
+            float d0, d1;
+            f32x2_split(d2, d0, d1);
+            ds[c2][c >> 1] = pack_bf16(d0, d1);
+          }
+      } else {                  // keys past the segment's end: S and dP hold anything, dS must be 0
+#pragma unroll
+        for (int c2 = 0; c2 < NL; ++c2)
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            const uint64_t d2 = mul2(p2[c2][c >> 1],
+                                     add2(f32x2(__uint_as_float(dp[c2][c]), __uint_as_float(dp[c2][c + 1])), nd2));
+            float d0, d1;
+            f32x2_split(d2, d0, d1);
             if (c2 * 32 + c >= valid) d0 = 0.f;
             if (c2 * 32 + c + 1 >= valid) d1 = 0.f;
+            ds[c2][c >> 1] = pack_bf16(d0, d1);
           }
-          ds[c2][c >> 1] = pack_bf16(d0, d1);
-        }
+      }
 #pragma unroll
       for (int c2 = 0; c2 < NL; ++c2)
         tmem_st16(tmem_lane + kColdS + g * (kDqCols / 2) + c2 * 16, ds[c2]);
