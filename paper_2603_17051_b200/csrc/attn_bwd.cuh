@@ -331,7 +331,7 @@ template <int D> struct DkvSmem {
   static constexpr int kV = TileGeom<D>::kBytes;
   static constexpr int kQ = 2 * TileGeom<D>::kBytes;                      // [kDkvStages]
   static constexpr int kdO = kQ + kDkvStages * TileGeom<D>::kBytes;       // [kDkvStages]
-  static constexpr int kStats = kdO + kDkvStages * TileGeom<D>::kBytes;   // float2 [2][128]: (lse*log2e, delta)
+  static constexpr int kStats = kdO + kDkvStages * TileGeom<D>::kBytes;   // float [stages][2][128]: -lse*log2e, -delta
   static constexpr int kBars = kStats + 2 * kTile * 8;
   static constexpr int kTotal = kBars + 256 + 1024;
 };
@@ -349,7 +349,7 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
   uint8_t* sV = smem + DkvSmem<D>::kV;
   uint8_t* sQ = smem + DkvSmem<D>::kQ;
   uint8_t* sdO = smem + DkvSmem<D>::kdO;
-  float2* sStat = reinterpret_cast<float2*>(smem + DkvSmem<D>::kStats);
+  float* sStat = reinterpret_cast<float*>(smem + DkvSmem<D>::kStats);   // [stage][-LSE*log2e | -delta][128 queries]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + DkvSmem<D>::kBars);
   uint64_t* kv_full = bars;
   uint64_t* q_full = bars + 1;                 // [kDkvStages]
@@ -410,12 +410,13 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         tma_load_tile<D>(sQ + st * TileGeom<D>::kBytes, &tm_q, q_full + st, i * kTile, h, b);
         tma_load_tile<D>(sdO + st * TileGeom<D>::kBytes, &tm_do, q_full + st, i * kTile, h, b);
       }
-      float2* stat = sStat + st * kTile;
+      float* stat = sStat + st * 2 * kTile;
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int qi = i * kTile + lane * 4 + e;
-        stat[lane * 4 + e] = qi < n_q ? make_float2(lse[stat_base + qi] * kLog2e, delta[stat_base + qi])
-                                      : make_float2(INFINITY, 0.f);
+        // negated once here, so that the consumers' loops add them as they come; +inf as LSE turns rows past n_q into P = 0
+        stat[lane * 4 + e] = qi < n_q ? -lse[stat_base + qi] * kLog2e : -INFINITY;
+        stat[kTile + lane * 4 + e] = qi < n_q ? -delta[stat_base + qi] : 0.f;
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(q_full + st);
@@ -464,7 +465,7 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     const uint64_t sc2 = f32x2(scale_log2, scale_log2);
     for (int i = 0; i < n_tiles; ++i) {
       // per-query constants of this group's 64 queries, staged by the producer warp with the tile
-      const float2* stat = sStat + (i % kDkvStages) * kTile + g * 64;
+      const float* stat = sStat + (i % kDkvStages) * 2 * kTile + g * 64;
       mbar_wait(q_full + i % kDkvStages, (i / kDkvStages) & 1, abort_flag);
       mbar_wait(s_full, i & 1, abort_flag);
       tc_fence_after_sync();
@@ -477,9 +478,8 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
       for (int c2 = 0; c2 < 2; ++c2)
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
-          const float4 st2 = *reinterpret_cast<const float4*>(stat + c2 * 32 + c);  // (lse2, delta) x 2 queries
-          const uint64_t x2 = fma2(f32x2(__uint_as_float(s[c2][c]), __uint_as_float(s[c2][c + 1])), sc2,
-                                   f32x2(-st2.x, -st2.z));
+          const uint64_t nl2 = *reinterpret_cast<const uint64_t*>(stat + c2 * 32 + c);   // -LSE*log2e of 2 queries
+          const uint64_t x2 = fma2(f32x2(__uint_as_float(s[c2][c]), __uint_as_float(s[c2][c + 1])), sc2, nl2);
           float p0, p1;
           if (((c >> 1) & 7) < kDkvPolyOf8) {
             exp2_poly_pair(x2, p0, p1);
@@ -507,9 +507,8 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
         tmem_wait_ld();
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
-          const float4 st2 = *reinterpret_cast<const float4*>(stat + c2 * 32 + c);
-          const uint64_t d2 = mul2(p2[c2][c >> 1], add2(f32x2(__uint_as_float(dp[c]), __uint_as_float(dp[c + 1])),
-                                                        f32x2(-st2.y, -st2.w)));
+          const uint64_t nd2 = *reinterpret_cast<const uint64_t*>(stat + kTile + c2 * 32 + c);   // -delta of 2 queries
+          const uint64_t d2 = mul2(p2[c2][c >> 1], add2(f32x2(__uint_as_float(dp[c]), __uint_as_float(dp[c + 1])), nd2));
           float d0, d1;
           f32x2_split(d2, d0, d1);
           ds[c >> 1] = pack_bf16(d0, d1);
