@@ -349,13 +349,13 @@ __device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdF
   const int g = warp >> 2;
   const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
   float m_ref = 0.f, l_run = 0.f, poly_max = -INFINITY;
-  int j = 0;
-  for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
-    const int valid = it.valid(segs) - kFwdCols * g;  // valid keys of this group's share (may be <= 0)
+  constexpr int NL = kFwdCols / 32;  // 32-column TMEM loads per thread and tile
+  // One key tile; `valid` = valid keys of this group's share (may be <= 0).  Full tiles pass the constant kFwdCols,
+  // so that nothing about key validity is left in their code.
+  auto tile = [&](int j, int valid) {
     const uint32_t colS = kFwdColS + (j % kFwdSBufs) * 128 + g * kFwdCols;
     mbar_wait(bar.sdone + j % 4, (j / 4) & 1, u.abort_flag);
     tc_fence_after_sync();
-    constexpr int NL = kFwdCols / 32;  // 32-column TMEM loads per thread and tile
     uint32_t s[NL][32];
 #pragma unroll
     for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);
@@ -387,6 +387,13 @@ __device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdF
     tmem_wait_st();
     tc_fence_before_sync();
     mbar_arrive(bar.ready + j % 4);
+  };
+  // key ranges one after the other: their full tiles in a loop of their own, then the ragged last tile if any
+  int j = 0;
+  for (int sg = 0; sg < segs.n; ++sg) {
+    const int full = segs.count[sg] / kTile, rest = segs.count[sg] % kTile;
+    for (int t = 0; t < full; ++t, ++j) tile(j, kFwdCols);
+    if (rest) { tile(j, rest - kFwdCols * g); ++j; }
   }
   bool ok = (l_run < kFastSumLimit) && !(poly_max > kPolyArgLimit);   // false for inf and NaN too
   ok = fwd_epilogue<D>(u, bar.o_full, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
