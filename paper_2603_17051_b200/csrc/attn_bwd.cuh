@@ -229,12 +229,12 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
       tc_fence_before_sync();
       mbar_arrive(qt_full);
     }
-    int j = 0;
-    for (KeyTileIter it; !it.done(segs); it.next(segs), ++j) {
-      const int valid = it.valid(segs) - kDqCols * g;  // valid keys of this group's share (may be <= 0)
+    constexpr int NL = kDqCols / 32;
+    // One key tile; `valid` = valid keys of this group's share (may be <= 0).  Full tiles pass the constant
+    // kDqCols, which leaves nothing about key validity in their code.
+    auto tile = [&](int j, int valid) {
       mbar_wait(s_full, j & 1, abort_flag);
       tc_fence_after_sync();
-      constexpr int NL = kDqCols / 32;
       uint32_t s[NL][32];
 #pragma unroll
       for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + kColS + g * kDqCols + c2 * 32, s[c2]);
@@ -297,6 +297,13 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(rb + j % 4);   // dS(j) stored; dP(j) was read before it, so its buffer is free as well
+    };
+    // key ranges one after the other: their full tiles in a loop of their own, then the ragged last tile if any
+    int j = 0;
+    for (int sg = 0; sg < segs.n; ++sg) {
+      const int full = segs.count[sg] / kTile, rest = segs.count[sg] % kTile;
+      for (int t = 0; t < full; ++t, ++j) tile(j, kDqCols);
+      if (rest) { tile(j, rest - kDqCols * g); ++j; }
     }
     // ---- epilogue: groups 0 and 1 write columns [g D/2, (g+1) D/2) of dQ
     mbar_wait(dq_full, 0, abort_flag);
