@@ -76,6 +76,21 @@ astro_status_t check_arch() {
   return ASTRO_OK;
 }
 
+// Number of SMs of the current device (0 if it cannot be read).
+int sm_count() {
+  static std::atomic<int> count[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (dev >= 0 && dev < kMaxDevices) {
+    const int c = count[dev].load(std::memory_order_acquire);
+    if (c > 0) return c;
+  }
+  int n = 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  if (dev >= 0 && dev < kMaxDevices) count[dev].store(n, std::memory_order_release);
+  return n;
+}
+
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -257,9 +272,16 @@ astro_status_t launch_fwd(const AttnArgs& a, const __nv_bfloat16* q, const CUten
   astro_status_t s = set_smem_once(chunk_attn_fwd_kernel<D>, FwdSmem<D>::kTotal, done);
   if (s != ASTRO_OK) return s;
   const int shared = (a.cache && a.cache->d.cache_batch == 1 && a.batch > 1) ? 1 : 0;
-  dim3 grid((a.n_q + kTile - 1) / kTile, shared ? a.batch : a.heads, shared ? a.heads : a.batch);
-  chunk_attn_fwd_kernel<D><<<grid, kFwdThreads, FwdSmem<D>::kTotal, st>>>(
-      q, tkc, tvc, tkx, tvx[0], tvx[1], segs, a.n_q, a.heads, shared,
+  // One CTA per SM, each walking over its share of the (query tile, head, sample) units; more CTAs only when a
+  // CTA would get more units than it has redo bits for.
+  const long long units = static_cast<long long>((a.n_q + kTile - 1) / kTile) * a.heads * a.batch;
+  const int sms = sm_count();
+  if (sms <= 0) return ASTRO_ERR_CUDA;
+  if (units > 0x7fffffffLL) return ASTRO_ERR_SHAPE;
+  long long ctas = units < sms ? units : sms;
+  if (units > ctas * kFwdMaxUnits) ctas = sms * ((units + static_cast<long long>(sms) * kFwdMaxUnits - 1) / (static_cast<long long>(sms) * kFwdMaxUnits));
+  chunk_attn_fwd_kernel<D><<<static_cast<unsigned>(ctas), kFwdThreads, FwdSmem<D>::kTotal, st>>>(
+      q, tkc, tvc, tkx, tvx[0], tvx[1], segs, a.batch, a.n_q, a.heads, shared,
       scale * kLog2e, g_fwd_mode.load(std::memory_order_relaxed) == 1 ? 1 : 0, static_cast<__nv_bfloat16*>(o), lse);
   return launch_status();
 }

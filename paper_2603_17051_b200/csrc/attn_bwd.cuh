@@ -158,7 +158,7 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
       load_kv(0, kv0_full, kv0_full);
       for (int t = 1; t <= n_tiles; ++t) {
         // commit t-1 of b_done: dQ(t-3) and dP(t-2) are done, the K stage and the V stage of tile t are free
-        if (t >= 2) mbar_wait_spin(b_done + ((t - 1) & 1), ((t - 2) >> 1) & 1, abort_flag);
+        if (t >= 2 && !mbar_wait_spin(b_done + ((t - 1) & 1), ((t - 2) >> 1) & 1, abort_flag)) break;
         if (t < n_tiles) {
           mbar_arrive_expect_tx(rs + (t - 1) % 4, TileGeom<D>::kBytes);
           mbar_arrive_expect_tx(rb + (t - 1) % 4, TileGeom<D>::kBytes);
@@ -314,6 +314,7 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
     }
   }
 
+  settle_after_abort(abort_flag);
   tc_fence_before_sync();
   __syncthreads();
   if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
@@ -411,8 +412,8 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     }
     for (int i = 0; i < n_tiles; ++i) {
       const int st = i % kDkvStages;
-      mbar_wait(q_empty + st, ((i / kDkvStages) & 1) ^ 1, abort_flag);
-      if (lane == 0) {
+      const bool go = mbar_wait(q_empty + st, ((i / kDkvStages) & 1) ^ 1, abort_flag);
+      if (lane == 0 && go) {   // no copies once a wait has run out
         mbar_arrive_expect_tx(q_full + st, 2 * TileGeom<D>::kBytes);
         tma_load_tile<D>(sQ + st * TileGeom<D>::kBytes, &tm_q, q_full + st, i * kTile, h, b);
         tma_load_tile<D>(sdO + st * TileGeom<D>::kBytes, &tm_do, q_full + st, i * kTile, h, b);
@@ -535,6 +536,7 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     store_row_from_tmem<D / 2>(tmem_lane + kColdV + g * (D / 2), 1.f, dv + row_off, in_range);
   }
 
+  settle_after_abort(abort_flag);
   tc_fence_before_sync();
   __syncthreads();
   if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);

@@ -24,8 +24,10 @@
 //   safe pass  only if some row of the CTA saw a sum beyond 2^100, an infinity or a NaN in the fast pass: the
 //              whole tile is recomputed with a running reference that follows the row maximum (rescaling O
 //              and the row sums when a tile's row sum leaves the safe range).
-//   TMEM columns: S buffers [0,128) [128,256)   O [256,256+D)   Q [384,384+D/2)
+//   TMEM columns: S buffers [0,128) [128,256)   O [256,256+D)   Q buffers [384,384+D/2) [448,448+D/2)
 #pragma once
+#include <type_traits>
+
 #include "attn_common.cuh"
 
 namespace astro {
@@ -35,13 +37,14 @@ constexpr int kFwdGroups = 4;                    // layer shape, forward alone: 
 constexpr int kFwdCols = kTile / kFwdGroups;     // keys per group and tile
 constexpr int kFwdThreads = 128 * kFwdGroups + 64;
 constexpr int kFwdBarSlots = 32;                 // mbarriers of one pass
+constexpr int kFwdMaxUnits = 1024;               // work units one CTA may walk (one redo bit each)
 
 template <int D> struct FwdSmem {
   static constexpr int kK = 0;
   static constexpr int kV = kK + kFwdKStages * TileGeom<D>::kBytes;
-  static constexpr int kMax = kV + kFwdVStages * TileGeom<D>::kBytes;  // float [2 parities + 1][groups][128]
-  static constexpr int kBars = kMax + 3 * kFwdGroups * kTile * 4;      // two sets of barriers, then 3 words
-  static constexpr int kTotal = kBars + 2 * kFwdBarSlots * 8 + 64 + 1024;  // + slack to align to 1024
+  static constexpr int kMax = kV + kFwdVStages * TileGeom<D>::kBytes;  // float [4][groups][128]: exchange slots
+  static constexpr int kBars = kMax + 4 * kFwdGroups * kTile * 4;      // two sets of barriers, 3 words, redo bits
+  static constexpr int kTotal = kBars + 2 * kFwdBarSlots * 8 + 64 + kFwdMaxUnits / 8 + 1024;  // + slack to align to 1024
 };
 
 // Of every 8 pairs of exponentials, how many use the polynomial on the FMA pipe.  Layer shape, forward alone:
@@ -71,12 +74,18 @@ struct FwdBars {
     mbar_init(pv_done + 1, 1);
     mbar_init(o_full, 1);
   }
+  // Fresh phases for another run of the pass; every thread of the CTA is past its last use of the barriers.
+  __device__ void rearm(int q_count, int p_count) const {
+    for (uint64_t* b = q_full; b <= o_full; ++b) mbar_inval(b);
+    init(q_count, p_count);
+  }
 };
 
 // What every role of the CTA needs to know about its work unit.
 template <int D> struct FwdUnit {
   const CUtensorMap *tm_kc, *tm_vc, *tm_kx;
-  const CUtensorMap* tm_vx[2];   // one per cache key range, each ending where its range ends (rows past it read as 0)
+  const CUtensorMap *tm_vx0, *tm_vx1;   // one per cache key range, each ending where its range ends (rows past it read as 0)
+  __device__ const CUtensorMap* vx(int seg) const { return seg == 0 ? tm_vx0 : tm_vx1; }
   const KeySegs* segs;
   uint8_t *sK, *sV;
   float* smax;
@@ -85,7 +94,8 @@ template <int D> struct FwdUnit {
   int n_tiles, h, b, bx;
 };
 
-constexpr uint32_t kFwdColS = 0 /* + 128 * buffer */, kFwdColO = 256, kFwdColQ = 384;
+constexpr uint32_t kFwdColS = 0 /* + 128 * buffer */, kFwdColO = 256, kFwdColQ = 384 /* + 64 * buffer */;
+constexpr uint32_t kFwdQCols = 64;
 
 // ---------------------------------------------------------------------------------- TMA producer (one thread)
 // K runs ahead of V by the S look-ahead: order the loads K0 K1 | V0 K2 | V1 K3 | ...
@@ -107,93 +117,189 @@ __device__ __forceinline__ void fwd_produce(const FwdUnit<D>& u, const FwdBars& 
     const bool fc = itv.from_chunk(segs);
     mbar_wait_spin(bar.v_empty + st, ((j / kFwdVStages) & 1) ^ 1, u.abort_flag);
     mbar_arrive_expect_tx(bar.v_full + st, TileGeom<D>::kBytes);
-    tma_load_tile<D>(u.sV + st * TileGeom<D>::kBytes, fc ? u.tm_vc : u.tm_vx[itv.seg], bar.v_full + st, itv.row0(segs), u.h,
+    tma_load_tile<D>(u.sV + st * TileGeom<D>::kBytes, fc ? u.tm_vc : u.vx(itv.seg), bar.v_full + st, itv.row0(segs), u.h,
                      fc ? u.b : u.bx);
     itv.next(segs);
   };
   for (int j = 0; j < kFwdSBufs && j < u.n_tiles; ++j) load_k(j);
   for (int j = 0; j < u.n_tiles; ++j) {
+    if (*u.abort_flag) break;
     load_v(j);
     if (j + kFwdSBufs < u.n_tiles) load_k(j + kFwdSBufs);
   }
 }
 
-// ---------------------------------------------------------------------------------- fast pass: barriers
-// The MMA-issuing thread is the pace-maker of the kernel, so the fast pass gives it ONE wait and ONE commit per key
-// tile.  ready[j % 4] collects everything tile j needs: the bytes of V(j) and K(j+2) (the producer's arrive with the
-// byte count plus the TMA completions) and the arrival of every softmax thread that has stored its P(j).
-// sdone[t % 4] is committed behind S(t): S(t) is ready for the softmax threads, and -- MMAs complete in order --
-// the P V of tile t-2 is done too, so the producer may refill the K stage of tile t and the V stage of tile t-2.
-struct FwdFastBars {
-  uint64_t *q_full, *k01, *ready, *sdone, *o_full;
-  __device__ explicit FwdFastBars(uint64_t* b) : q_full(b), k01(b + 1), ready(b + 2), sdone(b + 6), o_full(b + 10) {}
-  __device__ void init(int q_count) const {
-    mbar_init(q_full, q_count);
-    mbar_init(k01, 1);
-    for (int i = 0; i < 4; ++i) { mbar_init(ready + i, 1 + 128 * kFwdGroups); mbar_init(sdone + i, 1); }
-    mbar_init(o_full, 1);
+// ---------------------------------------------------------------------------------- fast pass: schedule
+// A CTA walks over work units (one 128-query tile of one head of one sample each): first, first + stride, ...
+// Unit ids count the query tiles fastest, then y, then z, where (y, z) = (head, sample), or (sample, head) when one
+// stored prefix serves every sample: then the samples of a head sit next to each other, and the CTAs that run at
+// the same time read the same cached K/V, which is fetched from HBM once and served out of L2.
+struct FwdSched {
+  int first, stride, total, q_tiles, dim_y, cache_shared;
+  __device__ int count() const { return (total - first + stride - 1) / stride; }
+  __device__ void decode(int unit, int& q_tile, int& h, int& b) const {
+    q_tile = unit % q_tiles;
+    const int yz = unit / q_tiles, y = yz % dim_y, z = yz / dim_y;
+    h = cache_shared ? z : y;
+    b = cache_shared ? y : z;
   }
 };
 
+// Position in the CTA's stream of key tiles: the tiles of its first unit, then those of the next, ...
+struct FwdCursor {
+  KeyTileIter it;
+  int unit, h, b, bx;
+  __device__ void set(const FwdSched& s) {
+    int qt;
+    s.decode(unit, qt, h, b);
+    bx = s.cache_shared ? 0 : b;
+  }
+  __device__ void start(const FwdSched& s) { unit = s.first; set(s); }
+  __device__ void next(const KeySegs& segs, const FwdSched& s) {
+    it.next(segs);
+    if (it.done(segs)) {
+      it = KeyTileIter();
+      unit += s.stride;
+      if (unit < s.total) set(s);
+    }
+  }
+};
+
+// ---------------------------------------------------------------------------------- fast pass: barriers
+// The MMA-issuing thread is the pace-maker of the kernel, so the fast pass gives it ONE wait and ONE commit per key
+// tile, and the key tiles of all the CTA's units form ONE stream (tile J of the stream; S two tiles ahead of P V
+// across unit boundaries as well), so the tensor pipe does not drain between units.
+// ready[J % 4] collects everything tile J needs: the bytes of V(J) and K(J+2) (the producer's arrive with the
+// byte count plus the TMA completions) and the arrival of every softmax thread that has stored its P(J).
+// sdone[J % 4] is committed behind S(J): S(J) is ready for the softmax threads, and -- MMAs complete in order --
+// the P V of tile J-2 is done too, so the producer may refill the K stage of tile J and the V stage of tile J-2.
+// Per unit: q_full[n % 2] (the unit's Q rows are in tensor memory buffer n % 2), o_full (its last P V is done),
+// o_free (every softmax thread has read its part of O: the next unit's first P V may overwrite it).
+struct FwdFastBars {
+  uint64_t *q_full, *k01, *ready, *sdone, *o_full, *o_free;
+  __device__ explicit FwdFastBars(uint64_t* b)
+      : q_full(b), k01(b + 2), ready(b + 3), sdone(b + 7), o_full(b + 11), o_free(b + 12) {}
+  __device__ void init(int q_count) const {
+    mbar_init(q_full, q_count);
+    mbar_init(q_full + 1, q_count);
+    mbar_init(k01, 1);
+    for (int i = 0; i < 4; ++i) { mbar_init(ready + i, 1 + 128 * kFwdGroups); mbar_init(sdone + i, 1); }
+    mbar_init(o_full, 1);
+    mbar_init(o_free, 128 * kFwdGroups);
+  }
+};
+
+// The loops of the three roles work from local copies of what they need: nothing in them reads `u`, `sch` or `bar`
+// again, whatever the compiler decides about where those structures live.
 template <int D>
-__device__ __forceinline__ void fwd_produce_fast(const FwdUnit<D>& u, const FwdFastBars& bar) {
+__device__ __forceinline__ void fwd_produce_fast(const FwdUnit<D>& u, const FwdSched& sch_in, const FwdFastBars& bar) {
   const KeySegs& segs = *u.segs;
-  KeyTileIter itk, itv;
-  auto load_k = [&](int j, uint64_t* full) {
-    const bool fc = itk.from_chunk(segs);
-    tma_load_tile<D>(u.sK + (j % kFwdKStages) * TileGeom<D>::kBytes, fc ? u.tm_kc : u.tm_kx, full, itk.row0(segs), u.h,
-                     fc ? u.b : u.bx);
-    itk.next(segs);
+  const FwdSched sch = sch_in;
+  const int total = u.n_tiles * sch.count();
+  const CUtensorMap *tm_kc = u.tm_kc, *tm_vc = u.tm_vc, *tm_kx = u.tm_kx, *tm_vx0 = u.tm_vx0, *tm_vx1 = u.tm_vx1;
+  uint8_t *sK = u.sK, *sV = u.sV;
+  uint64_t *ready = bar.ready, *sdone = bar.sdone;
+  volatile int* abort_flag = u.abort_flag;
+  FwdCursor ck, cv;   // K runs two tiles ahead of V
+  ck.start(sch);
+  cv.start(sch);
+  auto load_k = [&](int J, uint64_t* full) {
+    const bool fc = ck.it.from_chunk(segs);
+    tma_load_tile<D>(sK + (J % kFwdKStages) * TileGeom<D>::kBytes, fc ? tm_kc : tm_kx, full, ck.it.row0(segs),
+                     ck.h, fc ? ck.b : ck.bx);
+    ck.next(segs, sch);
   };
-  const int n01 = u.n_tiles < kFwdSBufs ? u.n_tiles : kFwdSBufs;
+  const int n01 = total < kFwdSBufs ? total : kFwdSBufs;
   mbar_arrive_expect_tx(bar.k01, n01 * TileGeom<D>::kBytes);
-  for (int j = 0; j < n01; ++j) load_k(j, bar.k01);
-  for (int j = 0; j < u.n_tiles; ++j) {
-    // S(j-1) done: the K stage of tile j+2 (that of tile j-1) and the V stage of tile j (that of tile j-3) are free
-    if (j >= 1) mbar_wait_spin(bar.sdone + (j - 1) % 4, ((j - 1) / 4) & 1, u.abort_flag);
-    const bool more = j + kFwdSBufs < u.n_tiles;
-    uint64_t* full = bar.ready + j % 4;
+  for (int J = 0; J < n01; ++J) load_k(J, bar.k01);
+  for (int J = 0; J < total; ++J) {
+    // S(J-1) done: the K stage of tile J+2 (that of tile J-1) and the V stage of tile J (that of tile J-3) are free
+    if (J >= 1 && !mbar_wait_spin(sdone + (J - 1) % 4, ((J - 1) / 4) & 1, abort_flag)) break;
+    const bool more = J + kFwdSBufs < total;
+    uint64_t* full = ready + J % 4;
     mbar_arrive_expect_tx(full, (more ? 2 : 1) * TileGeom<D>::kBytes);
-    const bool fc = itv.from_chunk(segs);
-    tma_load_tile<D>(u.sV + (j % kFwdVStages) * TileGeom<D>::kBytes, fc ? u.tm_vc : u.tm_vx[itv.seg], full,
-                     itv.row0(segs), u.h, fc ? u.b : u.bx);
-    itv.next(segs);
-    if (more) load_k(j + kFwdSBufs, full);
+    const bool fc = cv.it.from_chunk(segs);
+    tma_load_tile<D>(sV + (J % kFwdVStages) * TileGeom<D>::kBytes, fc ? tm_vc : (cv.it.seg == 0 ? tm_vx0 : tm_vx1), full,
+                     cv.it.row0(segs), cv.h, fc ? cv.b : cv.bx);
+    cv.next(segs, sch);
+    if (more) load_k(J + kFwdSBufs, full);
   }
 }
 
 template <int D>
-__device__ __forceinline__ void fwd_issue_fast(const FwdUnit<D>& u, const FwdFastBars& bar) {
+__device__ __forceinline__ void fwd_issue_fast(const FwdUnit<D>& u, const FwdSched& sch, const FwdFastBars& bar) {
   const uint64_t k_desc0 = desc_kmajor(smem_u32(u.sK));
+  const uint32_t sV_addr = smem_u32(u.sV);
   constexpr uint32_t idesc_s = make_idesc_bf16(kTile, kTile, false, false);
   constexpr uint32_t idesc_pv = make_idesc_bf16(kTile, D, false, true);
   const uint32_t tmem_base = u.tmem_base;
-  auto issue_s = [&](int j) {  // S(j) -> buffer j % 2; free because the PV of tile j-2 was issued before
-    const uint64_t k_desc = desc_step(k_desc0, (j % kFwdKStages) * TileGeom<D>::kBytes);
+  const int T = u.n_tiles, total = T * sch.count();
+  uint64_t *q_full = bar.q_full, *ready = bar.ready, *sdone = bar.sdone, *o_full = bar.o_full, *o_free = bar.o_free;
+  volatile int* abort_flag = u.abort_flag;
+  // S(J) -> buffer J % 2 (free: the P V of tile J-2 was issued before), from the Q buffer `qbuf`
+  auto issue_s = [&](int J, int qbuf) {
+    const uint32_t qcol = tmem_base + kFwdColQ + qbuf * kFwdQCols;
+    const uint64_t k_desc = desc_step(k_desc0, (J % kFwdKStages) * TileGeom<D>::kBytes);
 #pragma unroll
     for (int k = 0; k < D / 16; ++k)  // 16 elements of the head dimension = 8 packed Q columns
-      mma_ts(tmem_base + kFwdColS + (j % kFwdSBufs) * 128, tmem_base + kFwdColQ + k * 8,
+      mma_ts(tmem_base + kFwdColS + (J % kFwdSBufs) * 128, qcol + k * 8,
              desc_step(k_desc, (k >> 2) * TileGeom<D>::kBlockBytes + (k & 3) * 32), idesc_s, k > 0);
-    mma_commit(bar.sdone + j % 4);
+    mma_commit(sdone + J % 4);
   };
-  mbar_wait_spin(bar.q_full, 0, u.abort_flag);
-  mbar_wait_spin(bar.k01, 0, u.abort_flag);
-  tc_fence_after_sync();
-  for (int j = 0; j < kFwdSBufs && j < u.n_tiles; ++j) issue_s(j);
-  for (int j = 0; j < u.n_tiles; ++j) {
-    const uint32_t pcol = tmem_base + kFwdColS + (j % kFwdSBufs) * 128;
-    const uint64_t v_desc = desc_mnmajor(smem_u32(u.sV + (j % kFwdVStages) * TileGeom<D>::kBytes), TileGeom<D>::kBlockBytes);
-    mbar_wait_spin(bar.ready + j % 4, (j / 4) & 1, u.abort_flag);
-    tc_fence_after_sync();
+  // P V of tile J; `first`: the unit's first tile, which starts O afresh
+  auto issue_pv = [&](int J, bool first) {
+    const uint32_t pcol = tmem_base + kFwdColS + (J % kFwdSBufs) * 128;
+    const uint64_t v_desc = desc_mnmajor(sV_addr + (J % kFwdVStages) * TileGeom<D>::kBytes, TileGeom<D>::kBlockBytes);
 #pragma unroll
     for (int kb = 0; kb < kTile / 16; ++kb) {
       // P of 16 keys = 8 packed columns; group g's pairs start at its own S columns
       const uint32_t a = pcol + (kb * 16 / kFwdCols) * kFwdCols + (kb * 16 % kFwdCols) / 2;
-      mma_ts(tmem_base + kFwdColO, a, desc_step(v_desc, kb * 2048), idesc_pv, (j > 0 || kb > 0) ? 1u : 0u);
+      mma_ts(tmem_base + kFwdColO, a, desc_step(v_desc, kb * 2048), idesc_pv, (!first || kb > 0) ? 1u : 0u);
     }
-    if (j + kFwdSBufs < u.n_tiles) issue_s(j + kFwdSBufs);
+  };
+  // S of the stream's tile J, which may open a unit: then the unit's Q rows must be in tensor memory
+  int s_n = 0, s_t = 0;        // unit (counted within the CTA) and tile within it of the next S to issue
+  auto issue_s_checked = [&](int J) {
+    if (s_t == 0) {
+      mbar_wait_spin(q_full + (s_n & 1), (s_n >> 1) & 1, abort_flag);
+      tc_fence_after_sync();
+    }
+    issue_s(J, s_n & 1);
+    if (++s_t == T) { s_t = 0; ++s_n; }
+  };
+  mbar_wait_spin(bar.k01, 0, abort_flag);
+  tc_fence_after_sync();
+  for (int J = 0; J < kFwdSBufs && J < total; ++J) issue_s_checked(J);
+  int J = 0;
+  for (int n = 0; J < total; ++n) {
+    // first tile of the unit: the previous unit's O must have been read out
+    mbar_wait_spin(ready + J % 4, (J / 4) & 1, abort_flag);
+    if (n > 0) mbar_wait_spin(o_free, (n - 1) & 1, abort_flag);
+    tc_fence_after_sync();
+    issue_pv(J, true);
+    if (T == 1) mma_commit(o_full);
+    if (J + kFwdSBufs < total) issue_s_checked(J + kFwdSBufs);
+    ++J;
+    // interior tiles: S two tiles ahead stays inside the unit, nothing to check
+    for (int t = 1; t + kFwdSBufs < T; ++t, ++J) {
+      mbar_wait_spin(ready + J % 4, (J / 4) & 1, abort_flag);
+      tc_fence_after_sync();
+      issue_pv(J, false);
+      issue_s(J + kFwdSBufs, n & 1);
+    }
+    if (T > kFwdSBufs + 1) {   // what the interior loop issued: the unit's tiles 3 .. T-1, which end the unit
+      s_t += T - 1 - kFwdSBufs;
+      if (s_t >= T) { s_t -= T; ++s_n; }
+    }
+    // last tiles of the unit (not the first): their S look-ahead belongs to the next unit
+    for (int t = (T - kFwdSBufs > 1 ? T - kFwdSBufs : 1); t < T; ++t, ++J) {
+      mbar_wait_spin(ready + J % 4, (J / 4) & 1, abort_flag);
+      tc_fence_after_sync();
+      issue_pv(J, false);
+      if (t == T - 1) mma_commit(o_full);
+      if (J + kFwdSBufs < total) issue_s_checked(J + kFwdSBufs);
+    }
   }
-  mma_commit(bar.o_full);
 }
 
 // ---------------------------------------------------------------------------------- MMA issuer (one thread)
@@ -296,14 +402,26 @@ __device__ __forceinline__ float fwd_exp32(const uint32_t (&s)[32], int valid, f
 }
 
 // Epilogue shared by both passes: row sum = sum of the groups' partial sums; 32-column slices of the output
-// row are dealt round-robin to the groups.  Returns false if a stored value was not finite.
+// row are dealt round-robin to the groups.  The slices are read out of tensor memory first; `o_free`, if given,
+// gets this thread's arrival right after that (O may be overwritten from then on).  `ex` = [G][128] floats for the
+// exchange of the partial sums.  Returns false if a stored value was not finite.
 template <int D, int G = kFwdGroups>
-__device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_full, int g, int r, uint32_t tmem_lane,
+__device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_full, uint32_t o_parity,
+                                             uint64_t* o_free, float* ex, int g, int r, uint32_t tmem_lane,
                                              float m_run, float l_run, bool in_range, __nv_bfloat16* dst,
                                              float* lse_dst) {
-  mbar_wait(o_full, 0, u.abort_flag);
+  constexpr int kSlices = D / 32, kOwn = (kSlices + G - 1) / G;
+  mbar_wait(o_full, o_parity, u.abort_flag);
   tc_fence_after_sync();
-  float* ex = u.smax;  // free: the last exchange through it was consumed before the last P was published
+  uint32_t acc[kOwn][32];
+#pragma unroll
+  for (int i = 0; i < kOwn; ++i)
+    if (g + i * G < kSlices) tmem_ld32(tmem_lane + kFwdColO + (g + i * G) * 32, acc[i]);
+  tmem_wait_ld();
+  if (o_free != nullptr) {
+    tc_fence_before_sync();
+    mbar_arrive(o_free);
+  }
   ex[g * kTile + r] = l_run;
   named_barrier_sync(5, 128 * G);
   float l = 0.f;
@@ -312,25 +430,23 @@ __device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_fu
   const float inv_l = 1.f / l;
   uint32_t worst = 0;
 #pragma unroll
-  for (int c4 = 0; c4 < D / 32; ++c4) {
-    if (c4 % G != g) continue;
-    uint32_t acc[32];
-    tmem_ld32(tmem_lane + kFwdColO + c4 * 32, acc);
-    tmem_wait_ld();
+  for (int i = 0; i < kOwn; ++i) {
+    const int c4 = g + i * G;
+    if (c4 >= kSlices) continue;
 #pragma unroll
     for (int c = 0; c < 32; ++c) {
-      acc[c] = __float_as_uint(__uint_as_float(acc[c]) * inv_l);
-      worst = max(worst, acc[c] & 0x7fffffffu);
+      acc[i][c] = __float_as_uint(__uint_as_float(acc[i][c]) * inv_l);
+      worst = max(worst, acc[i][c] & 0x7fffffffu);
     }
     if (in_range) {
       uint4* out = reinterpret_cast<uint4*>(dst + c4 * 32);
 #pragma unroll
       for (int v = 0; v < 4; ++v) {
         uint4 w;
-        w.x = pack_bf16(__uint_as_float(acc[8 * v + 0]), __uint_as_float(acc[8 * v + 1]));
-        w.y = pack_bf16(__uint_as_float(acc[8 * v + 2]), __uint_as_float(acc[8 * v + 3]));
-        w.z = pack_bf16(__uint_as_float(acc[8 * v + 4]), __uint_as_float(acc[8 * v + 5]));
-        w.w = pack_bf16(__uint_as_float(acc[8 * v + 6]), __uint_as_float(acc[8 * v + 7]));
+        w.x = pack_bf16(__uint_as_float(acc[i][8 * v + 0]), __uint_as_float(acc[i][8 * v + 1]));
+        w.y = pack_bf16(__uint_as_float(acc[i][8 * v + 2]), __uint_as_float(acc[i][8 * v + 3]));
+        w.z = pack_bf16(__uint_as_float(acc[i][8 * v + 4]), __uint_as_float(acc[i][8 * v + 5]));
+        w.w = pack_bf16(__uint_as_float(acc[i][8 * v + 6]), __uint_as_float(acc[i][8 * v + 7]));
         out[v] = w;
       }
     }
@@ -339,65 +455,150 @@ __device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_fu
   return worst < 0x7f800000u;
 }
 
+// Where the rows of a unit go, and the 64 Q elements this thread stages for it.
+template <int D> struct FwdRow {
+  bool in_range;
+  __nv_bfloat16* dst;
+  float* lse_dst;
+  const uint4* q_src;   // elements [64 (warp / 4), +64) of the row; only meaningful for the staging warps
+  __device__ FwdRow(const FwdSched& sch, int unit, int r, int q_part, const __nv_bfloat16* q, int n_q, int heads,
+                    __nv_bfloat16* o, float* lse) {
+    int qt, h, b;
+    sch.decode(unit, qt, h, b);
+    const int row = qt * kTile + r;
+    in_range = row < n_q;
+    const size_t at = (static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h;
+    dst = o + at * D;
+    lse_dst = lse ? lse + (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0) : nullptr;
+    q_src = reinterpret_cast<const uint4*>(q + at * D + q_part * 64);
+  }
+  __device__ void load_q(uint32_t (&qr)[32]) const {
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+      const uint4 t = in_range ? q_src[v] : make_uint4(0, 0, 0, 0);
+      qr[4 * v] = t.x; qr[4 * v + 1] = t.y; qr[4 * v + 2] = t.z; qr[4 * v + 3] = t.w;
+    }
+  }
+};
+
 // ---------------------------------------------------------------------------------- softmax, fast pass
-// Returns false if the row must be redone by the safe pass.
+// What a softmax thread needs for one key tile of the fast pass.
+struct FwdTileCtx {
+  uint32_t tmem_lane;
+  int g, r, warp;
+  float scale_log2;
+  uint64_t *sdone, *ready;
+  volatile int* abort_flag;
+  float* mslot;   // [groups][128] floats for the exchange of the first tile's row maxima
+};
+
+// One key tile J of the CTA's stream; `valid` = valid keys of this group's share (may be <= 0).  Full tiles pass the
+// constant kFwdCols, so that nothing about key validity is left in their code.  kFirst: the unit's first tile, which
+// fixes the rows' reference.
+template <bool kFirst>
+__device__ __forceinline__ void fwd_fast_tile(const FwdTileCtx& c, int J, int valid, float& m_ref, float& l_run,
+                                              float& poly_max) {
+  constexpr int NL = kFwdCols / 32;  // 32-column TMEM loads per thread and tile
+  const uint32_t colS = kFwdColS + (J % kFwdSBufs) * 128 + c.g * kFwdCols;
+  mbar_wait(c.sdone + J % 4, (J / 4) & 1, c.abort_flag);
+  tc_fence_after_sync();
+  uint32_t s[NL][32];
+#pragma unroll
+  for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(c.tmem_lane + colS + c2 * 32, s[c2]);
+  tmem_wait_ld();
+  if (kFirst) {
+    // the row's one reference: the maximum of the first tile, agreed between the threads of the row
+    float mx = -INFINITY;
+#pragma unroll
+    for (int c2 = 0; c2 < NL; ++c2)
+#pragma unroll
+      for (int k = 0; k < 32; ++k)
+        if (c2 * 32 + k < valid) mx = fmaxf(mx, __uint_as_float(s[c2][k]));
+    c.mslot[c.g * kTile + c.r] = mx;
+    named_barrier_sync(1 + (c.warp & 3), 32 * kFwdGroups);
+#pragma unroll
+    for (int og = 0; og < kFwdGroups; ++og) mx = fmaxf(mx, c.mslot[og * kTile + c.r]);  // finite: >= 1 valid key
+    m_ref = mx * c.scale_log2;
+  }
+  const float neg_m = -m_ref;
+  // V rows past a key range's end never hold stale data here: the cache ranges' tensor maps end with the range,
+  // the chunk's with the chunk, and TMA fills what lies beyond with zeros
+#pragma unroll
+  for (int c2 = 0; c2 < NL; ++c2) {
+    uint32_t pk[16];
+    l_run += fwd_exp32(s[c2], valid - 32 * c2, c.scale_log2, neg_m, pk, poly_max);
+    tmem_st16(c.tmem_lane + colS + c2 * 16, pk);   // in place: this thread has read all of its S columns
+  }
+  tmem_wait_st();
+  tc_fence_before_sync();
+  mbar_arrive(c.ready + J % 4);
+}
+
+// Walks the CTA's units.  The epilogue of a unit (O out of tensor memory, normalised, stored) comes after the first
+// key tile of the NEXT unit, whose S was issued two tiles earlier: the P V of that tile is the only thing that has
+// to wait for the epilogue's reads.  The Q rows of the next unit go into the other Q buffer once the first tile of
+// the current unit is through (every S of the unit before, the buffer's last reader, is complete by then).
+// A unit one of whose rows must be redone by the safe pass gets its bit set in `redo_bits`.
 template <int D>
-__device__ __forceinline__ bool fwd_softmax_fast(const FwdUnit<D>& u, const FwdFastBars& bar, int warp, int r,
-                                                 float scale_log2, bool in_range, __nv_bfloat16* dst,
-                                                 float* lse_dst) {
+__device__ __forceinline__ void fwd_softmax_fast(const FwdUnit<D>& u, const FwdSched& sch, const FwdFastBars& bar,
+                                                 int warp, int r, float scale_log2, const __nv_bfloat16* q, int n_q,
+                                                 int heads, __nv_bfloat16* o, float* lse, uint32_t* redo_bits) {
   const KeySegs& segs = *u.segs;
   const int g = warp >> 2;
-  const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-  float m_ref = 0.f, l_run = 0.f, poly_max = -INFINITY;
-  constexpr int NL = kFwdCols / 32;  // 32-column TMEM loads per thread and tile
-  // One key tile; `valid` = valid keys of this group's share (may be <= 0).  Full tiles pass the constant kFwdCols,
-  // so that nothing about key validity is left in their code.
-  auto tile = [&](int j, int valid) {
-    const uint32_t colS = kFwdColS + (j % kFwdSBufs) * 128 + g * kFwdCols;
-    mbar_wait(bar.sdone + j % 4, (j / 4) & 1, u.abort_flag);
-    tc_fence_after_sync();
-    uint32_t s[NL][32];
-#pragma unroll
-    for (int c2 = 0; c2 < NL; ++c2) tmem_ld32(tmem_lane + colS + c2 * 32, s[c2]);
-    tmem_wait_ld();
-    if (j == 0) {
-      // the row's one reference: the maximum of the first tile, agreed between the threads of the row
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c2 = 0; c2 < NL; ++c2)
-#pragma unroll
-        for (int c = 0; c < 32; ++c)
-          if (c2 * 32 + c < valid) mx = fmaxf(mx, __uint_as_float(s[c2][c]));
-      float* mslot = u.smax + 2 * kFwdGroups * kTile;
-      mslot[g * kTile + r] = mx;
-      named_barrier_sync(1 + (warp & 3), 32 * kFwdGroups);
-#pragma unroll
-      for (int og = 0; og < kFwdGroups; ++og) mx = fmaxf(mx, mslot[og * kTile + r]);  // finite: >= 1 valid key
-      m_ref = mx * scale_log2;
-    }
-    const float neg_m = -m_ref;
-    // V rows past a key range's end never hold stale data here: the cache ranges' tensor maps end with the range,
-    // the chunk's with the chunk, and TMA fills what lies beyond with zeros
-#pragma unroll
-    for (int c2 = 0; c2 < NL; ++c2) {
-      uint32_t pk[16];
-      l_run += fwd_exp32(s[c2], valid - 32 * c2, scale_log2, neg_m, pk, poly_max);
-      tmem_st16(tmem_lane + colS + c2 * 16, pk);   // in place: this thread has read all of its S columns
-    }
-    tmem_wait_st();
-    tc_fence_before_sync();
-    mbar_arrive(bar.ready + j % 4);
+  const bool stages_q = g < D / 64;
+  FwdTileCtx c;
+  c.tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+  c.g = g; c.r = r; c.warp = warp;
+  c.scale_log2 = scale_log2;
+  c.sdone = bar.sdone; c.ready = bar.ready;
+  c.abort_flag = u.abort_flag;
+  // the epilogue of the unit before (unit `unit`, the CTA's n-th), whose reference, row sum and verdict are kept
+  float m_prev = 0.f, l_prev = 0.f;
+  bool ok_prev = true;
+  auto finish = [&](int unit, int n) {
+    const FwdRow<D> row(sch, unit, r, g, q, n_q, heads, o, lse);
+    float* ex = u.smax + (n & 1) * kFwdGroups * kTile;   // alternates: a fast thread may be a unit ahead
+    const bool fin = fwd_epilogue<D>(u, bar.o_full, n & 1, bar.o_free, ex, g, r, c.tmem_lane, m_prev, l_prev,
+                                     row.in_range, row.dst, row.lse_dst);
+    if (!(fin && ok_prev)) atomicOr(redo_bits + (n >> 5), 1u << (n & 31));
   };
-  // key ranges one after the other: their full tiles in a loop of their own, then the ragged last tile if any
-  int j = 0;
-  for (int sg = 0; sg < segs.n; ++sg) {
-    const int full = segs.count[sg] / kTile, rest = segs.count[sg] % kTile;
-    for (int t = 0; t < full; ++t, ++j) tile(j, kFwdCols);
-    if (rest) { tile(j, rest - kFwdCols * g); ++j; }
+  const int c0 = segs.count[0], T = u.n_tiles;
+  int n = 0;
+  for (int unit = sch.first; unit < sch.total; unit += sch.stride, ++n) {
+    const bool has_next = unit + sch.stride < sch.total;
+    const int J = n * T;
+    float m_ref = 0.f, l_run = 0.f, poly_max = -INFINITY;
+    c.mslot = u.smax + (2 + (n & 1)) * kFwdGroups * kTile;   // alternates for the same reason
+    // where the next unit's Q rows are: worked out and asked for (into L2) now, fetched after the first tile
+    const FwdRow<D> next_row(sch, has_next ? unit + sch.stride : unit, r, g, q, n_q, heads, o, lse);
+    if (has_next && stages_q && next_row.in_range) prefetch_l2(next_row.q_src);
+    if (c0 >= kTile) fwd_fast_tile<true>(c, J, kFwdCols, m_ref, l_run, poly_max);
+    else fwd_fast_tile<true>(c, J, c0 - kFwdCols * g, m_ref, l_run, poly_max);
+    if (n > 0) finish(unit - sch.stride, n - 1);
+    if (has_next && stages_q) {
+      uint32_t qr[32];
+      next_row.load_q(qr);
+      tmem_st32(c.tmem_lane + kFwdColQ + ((n + 1) & 1) * kFwdQCols + g * 32, qr);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(bar.q_full + ((n + 1) & 1));
+    }
+    // the other tiles: key ranges one after the other, their full tiles in a loop of their own, then the ragged
+    // last tile if any
+    int Jr = J + 1;
+    for (int sg = 0; sg < segs.n; ++sg) {
+      int full = segs.count[sg] / kTile, rest = segs.count[sg] % kTile;
+      if (sg == 0) {   // minus the first tile
+        if (full > 0) --full; else rest = 0;
+      }
+      for (int t = 0; t < full; ++t, ++Jr) fwd_fast_tile<false>(c, Jr, kFwdCols, m_ref, l_run, poly_max);
+      if (rest) { fwd_fast_tile<false>(c, Jr, rest - kFwdCols * g, m_ref, l_run, poly_max); ++Jr; }
+    }
+    ok_prev = (l_run < kFastSumLimit) && !(poly_max > kPolyArgLimit);   // false for inf and NaN too
+    m_prev = m_ref;
+    l_prev = l_run;
   }
-  bool ok = (l_run < kFastSumLimit) && !(poly_max > kPolyArgLimit);   // false for inf and NaN too
-  ok = fwd_epilogue<D>(u, bar.o_full, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
-  return ok;
+  finish(sch.first + (n - 1) * sch.stride, n - 1);
 }
 
 // ---------------------------------------------------------------------------------- softmax, safe pass
@@ -507,15 +708,32 @@ __device__ __forceinline__ void fwd_softmax_safe(const FwdUnit<D>& u, const FwdB
     tc_fence_before_sync();
     mbar_arrive(bar.p_full + g * kFwdSBufs + buf);
   }
-  fwd_epilogue<D>(u, bar.o_full, g, r, tmem_lane, m_run, l_run, in_range, dst, lse_dst);
+  fwd_epilogue<D>(u, bar.o_full, 0, nullptr, u.smax, g, r, tmem_lane, m_run, l_run, in_range, dst, lse_dst);
 }
 
+// The safe pass of one unit, all roles.  Kept out of line: it is the rare path, and the registers it needs must not
+// weigh on the allocation of the fast pass around it.
+template <int D>
+__device__ __noinline__ void fwd_safe_unit(const FwdUnit<D>& u, const FwdBars& bar, int warp, int lane, int r,
+                                           float scale_log2, bool in_range, __nv_bfloat16* dst, float* lse_dst) {
+  constexpr int kMmaWarp = 4 * kFwdGroups, kTmaWarp = 4 * kFwdGroups + 1;
+  if (warp == kTmaWarp) {
+    if (lane == 0) fwd_produce<D>(u, bar);
+  } else if (warp == kMmaWarp) {
+    if (lane == 0) fwd_issue<D>(u, bar);
+  } else {
+    fwd_softmax_safe<D>(u, bar, warp, r, scale_log2, in_range, dst, lse_dst);
+  }
+}
+
+// grid.x CTAs share `batch * heads * ceil(n_q / 128)` work units (at most kFwdMaxUnits each): CTA i takes units
+// i, i + grid.x, ...  Launched with one CTA per SM the CTAs are all resident and each streams through its units.
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant__ CUtensorMap tm_kc,
                       const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kx,
                       const __grid_constant__ CUtensorMap tm_vx0, const __grid_constant__ CUtensorMap tm_vx1,
-                      const __grid_constant__ KeySegs segs, const int n_q,
+                      const __grid_constant__ KeySegs segs, const int batch, const int n_q,
                       const int heads, const int cache_shared, const float scale_log2, const int force_safe,
                       __nv_bfloat16* __restrict__ o, float* __restrict__ lse) {
   extern __shared__ uint8_t smem_raw[];
@@ -525,31 +743,26 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   const FwdBars bar_safe(bar_mem + kFwdBarSlots);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bar_mem + 2 * kFwdBarSlots);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
-  volatile int* redo_flag = reinterpret_cast<volatile int*>(tmem_holder + 2);
+  uint32_t* redo_bits = tmem_holder + 16;   // one bit per unit of this CTA
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // With one shared cache (frozen prefix of a sample group) the samples of a head are launched next to each
-  // other, so the head's cached K/V is fetched from HBM once and served to the whole group out of L2.
-  const int q0 = blockIdx.x * kTile;
-  const int h = cache_shared ? blockIdx.z : blockIdx.y, b = cache_shared ? blockIdx.y : blockIdx.z;
   constexpr uint32_t kTmemCols = 512;
   constexpr int kMmaWarp = 4 * kFwdGroups, kTmaWarp = 4 * kFwdGroups + 1;
+  FwdSched sch;
+  sch.q_tiles = (n_q + kTile - 1) / kTile;
+  sch.dim_y = cache_shared ? batch : heads;
+  sch.cache_shared = cache_shared;
+  sch.first = blockIdx.x;
+  sch.stride = gridDim.x;
+  sch.total = sch.q_tiles * heads * batch;
 
-  // Each softmax thread fetches its share of the Q row (64 elements: group g takes elements [64 g, 64 g + 64)) before
-  // anything else, so that the load's latency passes behind the barrier set-up and the tensor-memory allocation.
+  // Each softmax thread fetches its share of the first unit's Q row (64 elements: group g takes elements
+  // [64 g, 64 g + 64)) before anything else, so that the load's latency passes behind the barrier set-up and the
+  // tensor-memory allocation.
   const int r = tid & 127;           // query row inside the tile = TMEM lane (softmax warps)
-  const int row = q0 + r;
-  const bool in_range = row < n_q;
   const bool stages_q = warp < kMmaWarp && (warp >> 2) < D / 64;
   uint32_t qr[32];
-  if (stages_q) {
-    const uint4* src = reinterpret_cast<const uint4*>(q + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + (warp >> 2) * 64);
-#pragma unroll
-    for (int v = 0; v < 8; ++v) {
-      const uint4 t = in_range ? src[v] : make_uint4(0, 0, 0, 0);
-      qr[4 * v] = t.x; qr[4 * v + 1] = t.y; qr[4 * v + 2] = t.z; qr[4 * v + 3] = t.w;
-    }
-  }
+  if (stages_q && !force_safe) FwdRow<D>(sch, sch.first, r, warp >> 2, q, n_q, heads, o, lse).load_q(qr);
   if (warp == kTmaWarp && lane == 0) {
     tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc); tma_prefetch_desc(&tm_kx); tma_prefetch_desc(&tm_vx0);
   }
@@ -557,10 +770,10 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
     bar_fast.init(128 * (D / 64));  // q_full: the threads that write Q into tensor memory
     bar_safe.init(1, 128);
     *abort_flag = 0;
-    *redo_flag = force_safe;
     fence_mbar_init();
     fence_proxy_async_smem();
   }
+  if (tid < kFwdMaxUnits / 32) redo_bits[tid] = 0;
   if (warp == kMmaWarp) {
     tmem_alloc(tmem_holder, kTmemCols);
     tmem_relinquish();
@@ -570,7 +783,7 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   tc_fence_after_sync();
 
   FwdUnit<D> u;
-  u.tm_kc = &tm_kc; u.tm_vc = &tm_vc; u.tm_kx = &tm_kx; u.tm_vx[0] = &tm_vx0; u.tm_vx[1] = &tm_vx1;
+  u.tm_kc = &tm_kc; u.tm_vc = &tm_vc; u.tm_kx = &tm_kx; u.tm_vx0 = &tm_vx0; u.tm_vx1 = &tm_vx1;
   u.segs = &segs;
   u.sK = smem + FwdSmem<D>::kK;
   u.sV = smem + FwdSmem<D>::kV;
@@ -578,44 +791,58 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   u.abort_flag = abort_flag;
   u.tmem_base = *tmem_holder;
   u.n_tiles = seg_tiles(segs);
-  u.h = h; u.b = b; u.bx = cache_shared ? 0 : b;
+  u.h = u.b = u.bx = 0;   // set per unit by the safe pass; the fast pass follows its cursors
+  const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
 
-  __nv_bfloat16* dst = o + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D;
-  float* lse_dst = lse ? lse + (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0) : nullptr;
-
-  // ---- fast pass
-  if (warp == kTmaWarp) {
-    if (lane == 0 && !force_safe) fwd_produce_fast<D>(u, bar_fast);
-  } else if (warp == kMmaWarp) {
-    if (lane == 0 && !force_safe) fwd_issue_fast<D>(u, bar_fast);
-  } else {
-    // Q row -> tensor memory (32 packed columns per 64 elements)
-    const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-    if (stages_q) {
-      tmem_st32(tmem_lane + kFwdColQ + (warp >> 2) * 32, qr);
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(bar_fast.q_full);
+  // ---- fast pass over all the CTA's units
+  if (!force_safe) {
+    if (warp == kTmaWarp) {
+      if (lane == 0) fwd_produce_fast<D>(u, sch, bar_fast);
+    } else if (warp == kMmaWarp) {
+      if (lane == 0) fwd_issue_fast<D>(u, sch, bar_fast);
+    } else {
+      // Q row of the first unit -> tensor memory buffer 0 (32 packed columns per 64 elements)
+      if (stages_q) {
+        tmem_st32(tmem_lane + kFwdColQ + (warp >> 2) * 32, qr);
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(bar_fast.q_full);
+      }
+      fwd_softmax_fast<D>(u, sch, bar_fast, warp, r, scale_log2, q, n_q, heads, o, lse, redo_bits);
     }
-    if (!force_safe && !fwd_softmax_fast<D>(u, bar_fast, warp, r, scale_log2, in_range, dst, lse_dst)) *redo_flag = 1;
   }
 
-  // ---- safe pass, for the whole CTA, if any of its rows asked for it (every MMA of the fast pass has
-  //      finished by now: the softmax threads waited for the last one before their epilogue)
-  tc_fence_before_sync();
-  __syncthreads();
-  tc_fence_after_sync();
-  if (*redo_flag && !*abort_flag) {
-    if (warp == kTmaWarp) {
-      if (lane == 0) fwd_produce<D>(u, bar_safe);
-    } else if (warp == kMmaWarp) {
-      if (lane == 0) fwd_issue<D>(u, bar_safe);
-    } else {
-      fwd_softmax_safe<D>(u, bar_safe, warp, r, scale_log2, in_range, dst, lse_dst);
+  // ---- safe pass, unit by unit, for the units one of whose rows asked for it (every MMA of the fast pass has
+  //      finished by now: the softmax threads waited for the last one before their last epilogue)
+  int n = 0;
+  for (int unit = sch.first; unit < sch.total; unit += sch.stride, ++n) {
+    tc_fence_before_sync();
+    __syncthreads();   // the fast pass, or the unit before, is over for every thread: redo bits and barriers at rest
+    tc_fence_after_sync();
+    if (*abort_flag) break;
+    if (!force_safe && !((redo_bits[n >> 5] >> (n & 31)) & 1u)) continue;
+    int qt;
+    sch.decode(unit, qt, u.h, u.b);
+    u.bx = cache_shared ? 0 : u.b;
+    const FwdRow<D> row(sch, unit, r, warp >> 2, q, n_q, heads, o, lse);
+    if (tid == 0) {
+      bar_safe.rearm(1, 128);
+      fence_mbar_init();
+    }
+    if (stages_q) {
+      row.load_q(qr);
+      tmem_st32(tmem_lane + kFwdColQ + (warp >> 2) * 32, qr);
+      tmem_wait_st();
     }
     tc_fence_before_sync();
     __syncthreads();
+    tc_fence_after_sync();
+    const FwdUnit<D> su = u;   // a copy: `u` itself never leaves the registers of the fast pass
+    fwd_safe_unit<D>(su, bar_safe, warp, lane, r, scale_log2, row.in_range, row.dst, row.lse_dst);
   }
+  settle_after_abort(abort_flag);
+  tc_fence_before_sync();
+  __syncthreads();
   if (warp == kMmaWarp) tmem_dealloc(u.tmem_base, kTmemCols);
 }
 

@@ -131,6 +131,7 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
       };
       for (int j = 0; j < kFwdSBufs && j < n_tiles; ++j) load_k(j);
       for (int j = 0; j < n_tiles; ++j) {
+        if (*abort_flag) break;
         load_v(j);
         if (j + kFwdSBufs < n_tiles) load_k(j + kFwdSBufs);
       }
@@ -244,10 +245,11 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
     u.abort_flag = abort_flag;
     __nv_bfloat16* dst = o + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D;
     float* lse_dst = lse ? lse + (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0) : nullptr;
-    ok = fwd_epilogue<D, kPairGroups>(u, bar.o_full, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
+    ok = fwd_epilogue<D, kPairGroups>(u, bar.o_full, 0, nullptr, u.smax, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
     if (!ok) *needs_safe = 1;
   }
 
+  settle_after_abort(abort_flag);
   tc_fence_before_sync();
   __syncthreads();
   cluster_sync_all();              // the peer may still read this CTA's shared memory and arrive on its barriers
