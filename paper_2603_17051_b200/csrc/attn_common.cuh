@@ -36,6 +36,62 @@ struct KeyTileIter {
   }
 };
 
+// Rows of a row-major tensor seen by a warp whose lane L owns row L of 32 consecutive rows: the four lanes of a quad
+// (lanes 4m .. 4m+3) move the 64-byte pieces of their four rows together, each lane one 16-byte chunk of every row,
+// so that one warp-wide access touches 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes.
+// transpose4x4 turns "lane l of the quad holds chunks 0..3 of row l" into "lane l holds chunk l of rows 0..3"
+// (slot j = row j), and back: the exchange is its own inverse.
+__device__ __forceinline__ void quad_exchange(uint4& a, uint4& b, bool bit, int mask) {
+  // lanes with the bit clear keep a and swap b for the partner's a; lanes with it set keep b and swap a
+  const uint4 send = bit ? a : b;
+  uint4 recv;
+  recv.x = __shfl_xor_sync(0xffffffffu, send.x, mask);
+  recv.y = __shfl_xor_sync(0xffffffffu, send.y, mask);
+  recv.z = __shfl_xor_sync(0xffffffffu, send.z, mask);
+  recv.w = __shfl_xor_sync(0xffffffffu, send.w, mask);
+  if (bit) a = recv; else b = recv;
+}
+__device__ __forceinline__ void transpose4x4(uint4 (&c)[4], int lane) {
+  const bool b0 = lane & 1, b1 = lane & 2;
+  quad_exchange(c[0], c[1], b0, 1);
+  quad_exchange(c[2], c[3], b0, 1);
+  quad_exchange(c[0], c[2], b1, 2);
+  quad_exchange(c[1], c[3], b1, 2);
+}
+
+// The four rows of a lane's quad in a [.., rows, heads, D] bf16 tensor: `first` points at element 0 of the quad's
+// first row (for the head and sample at hand), rows are `stride` elements apart, `valid` of the four exist.
+struct QuadRows {
+  __nv_bfloat16* first;
+  size_t stride;
+  int valid;
+};
+__device__ __forceinline__ QuadRows quad_rows(const __nv_bfloat16* base, int b, int h, int n_rows, int heads, int D,
+                                              int own_row) {
+  QuadRows q;
+  const int row_first = own_row & ~3;
+  q.stride = static_cast<size_t>(heads) * D;
+  q.first = const_cast<__nv_bfloat16*>(base) + (static_cast<size_t>(b) * n_rows + row_first) * q.stride +
+            static_cast<size_t>(h) * D;
+  q.valid = n_rows - row_first;   // may be <= 0 or > 4
+  return q;
+}
+// Lane L holds 32 bf16 (64 bytes, as 4 chunks) of row L, destined for columns [col0, col0 + 32) of its row.
+__device__ __forceinline__ void store_quad_rows(uint4 (&c)[4], const QuadRows& q, int col0, int lane) {
+  transpose4x4(c, lane);
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    if (j < q.valid) *reinterpret_cast<uint4*>(q.first + j * q.stride + col0 + (lane & 3) * 8) = c[j];
+}
+// The reverse: 32 bf16 of columns [col0, col0 + 32) of the lane's own row (zeros for rows that do not exist).
+__device__ __forceinline__ void load_quad_rows(uint4 (&c)[4], const QuadRows& q, int col0, int lane) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    c[j] = j < q.valid ? *reinterpret_cast<const uint4*>(q.first + j * q.stride + col0 + (lane & 3) * 8)
+                       : make_uint4(0, 0, 0, 0);
+  transpose4x4(c, lane);
+}
+
 // A [128 x D] bf16 tile sits in shared memory as D/64 blocks of [128 rows x 128 bytes], 128-byte
 // swizzled by TMA; block h holds columns 64h..64h+63.
 template <int D> struct TileGeom {

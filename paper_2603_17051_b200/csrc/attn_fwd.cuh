@@ -145,6 +145,42 @@ struct FwdSched {
   }
 };
 
+// A unit as (query tile, y, z), stepped from one unit of the CTA to the next or the previous one without divisions.
+struct FwdPos {
+  int qt, y, z;
+  int dq, dy, dz;   // the CTA's stride, taken apart the same way
+  __device__ FwdPos(const FwdSched& s, int unit) {
+    qt = unit % s.q_tiles;
+    const int yz = unit / s.q_tiles;
+    y = yz % s.dim_y;
+    z = yz / s.dim_y;
+    dq = s.stride % s.q_tiles;
+    const int syz = s.stride / s.q_tiles;
+    dy = syz % s.dim_y;
+    dz = syz / s.dim_y;
+  }
+  __device__ void forward(const FwdSched& s) {
+    qt += dq;
+    int carry = 0;
+    if (qt >= s.q_tiles) { qt -= s.q_tiles; carry = 1; }
+    y += dy + carry;
+    carry = 0;
+    if (y >= s.dim_y) { y -= s.dim_y; carry = 1; }
+    z += dz + carry;
+  }
+  __device__ void back(const FwdSched& s) {
+    qt -= dq;
+    int borrow = 0;
+    if (qt < 0) { qt += s.q_tiles; borrow = 1; }
+    y -= dy + borrow;
+    borrow = 0;
+    if (y < 0) { y += s.dim_y; borrow = 1; }
+    z -= dz + borrow;
+  }
+  __device__ int h(const FwdSched& s) const { return s.cache_shared ? z : y; }
+  __device__ int b(const FwdSched& s) const { return s.cache_shared ? y : z; }
+};
+
 // Position in the CTA's stream of key tiles: the tiles of its first unit, then those of the next, ...
 struct FwdCursor {
   KeyTileIter it;
@@ -404,11 +440,12 @@ __device__ __forceinline__ float fwd_exp32(const uint32_t (&s)[32], int valid, f
 // Epilogue shared by both passes: row sum = sum of the groups' partial sums; 32-column slices of the output
 // row are dealt round-robin to the groups.  The slices are read out of tensor memory first; `o_free`, if given,
 // gets this thread's arrival right after that (O may be overwritten from then on).  `ex` = [G][128] floats for the
-// exchange of the partial sums.  Returns false if a stored value was not finite.
+// exchange of the partial sums.  The quads of a warp store their rows together (64 contiguous bytes per row).
+// Returns false if a stored value was not finite.
 template <int D, int G = kFwdGroups>
 __device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_full, uint32_t o_parity,
                                              uint64_t* o_free, float* ex, int g, int r, uint32_t tmem_lane,
-                                             float m_run, float l_run, bool in_range, __nv_bfloat16* dst,
+                                             float m_run, float l_run, const QuadRows& out, bool in_range,
                                              float* lse_dst) {
   constexpr int kSlices = D / 32, kOwn = (kSlices + G - 1) / G;
   mbar_wait(o_full, o_parity, u.abort_flag);
@@ -428,56 +465,74 @@ __device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_fu
 #pragma unroll
   for (int og = 0; og < G; ++og) l += ex[og * kTile + r];
   const float inv_l = 1.f / l;
-  uint32_t worst = 0;
+  const uint64_t inv2 = f32x2(inv_l, inv_l), zero2 = f32x2(0.f, 0.f);
+  uint64_t chk2 = zero2;   // stays 0 while every value times 0 is 0, i.e. while every value is finite
 #pragma unroll
   for (int i = 0; i < kOwn; ++i) {
     const int c4 = g + i * G;
-    if (c4 >= kSlices) continue;
+    if (c4 >= kSlices) continue;   // the same for the whole warp
+    uint4 ch[4];
 #pragma unroll
-    for (int c = 0; c < 32; ++c) {
-      acc[i][c] = __float_as_uint(__uint_as_float(acc[i][c]) * inv_l);
-      worst = max(worst, acc[i][c] & 0x7fffffffu);
-    }
-    if (in_range) {
-      uint4* out = reinterpret_cast<uint4*>(dst + c4 * 32);
+    for (int v = 0; v < 4; ++v) {
+      uint32_t w[4];
 #pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        uint4 w;
-        w.x = pack_bf16(__uint_as_float(acc[i][8 * v + 0]), __uint_as_float(acc[i][8 * v + 1]));
-        w.y = pack_bf16(__uint_as_float(acc[i][8 * v + 2]), __uint_as_float(acc[i][8 * v + 3]));
-        w.z = pack_bf16(__uint_as_float(acc[i][8 * v + 4]), __uint_as_float(acc[i][8 * v + 5]));
-        w.w = pack_bf16(__uint_as_float(acc[i][8 * v + 6]), __uint_as_float(acc[i][8 * v + 7]));
-        out[v] = w;
+      for (int e = 0; e < 4; ++e) {
+        const uint64_t f2 = mul2(f32x2(__uint_as_float(acc[i][8 * v + 2 * e]), __uint_as_float(acc[i][8 * v + 2 * e + 1])), inv2);
+        chk2 = fma2(f2, zero2, chk2);
+        float f0, f1;
+        f32x2_split(f2, f0, f1);
+        w[e] = pack_bf16(f0, f1);
       }
+      ch[v] = make_uint4(w[0], w[1], w[2], w[3]);
     }
+    store_quad_rows(ch, out, c4 * 32, r & 31);
   }
-  if (g == 0 && in_range && lse_dst != nullptr) *lse_dst = (m_run + log2f(l)) * 0.6931471805599453f;
-  return worst < 0x7f800000u;
+  if (g == G - 1 && in_range && lse_dst != nullptr) *lse_dst = (m_run + log2f(l)) * 0.6931471805599453f;
+  float chk0, chk1;
+  f32x2_split(chk2, chk0, chk1);
+  return chk0 == 0.f && chk1 == 0.f;
 }
 
-// Where the rows of a unit go, and the 64 Q elements this thread stages for it.
+// Where the rows of a unit are: the lane's own row for LSE, its quad's rows for O and Q.
 template <int D> struct FwdRow {
   bool in_range;
-  __nv_bfloat16* dst;
   float* lse_dst;
-  const uint4* q_src;   // elements [64 (warp / 4), +64) of the row; only meaningful for the staging warps
-  __device__ FwdRow(const FwdSched& sch, int unit, int r, int q_part, const __nv_bfloat16* q, int n_q, int heads,
+  QuadRows out, q_rows;
+  __device__ FwdRow(const FwdSched& sch, int unit, int r, const __nv_bfloat16* q, int n_q, int heads,
                     __nv_bfloat16* o, float* lse) {
     int qt, h, b;
     sch.decode(unit, qt, h, b);
+    init(qt, h, b, r, q, n_q, heads, o, lse);
+  }
+  __device__ FwdRow(const FwdSched& sch, const FwdPos& pos, int r, const __nv_bfloat16* q, int n_q, int heads,
+                    __nv_bfloat16* o, float* lse) {
+    init(pos.qt, pos.h(sch), pos.b(sch), r, q, n_q, heads, o, lse);
+  }
+  __device__ void init(int qt, int h, int b, int r, const __nv_bfloat16* q, int n_q, int heads, __nv_bfloat16* o,
+                       float* lse) {
     const int row = qt * kTile + r;
     in_range = row < n_q;
-    const size_t at = (static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h;
-    dst = o + at * D;
     lse_dst = lse ? lse + (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0) : nullptr;
-    q_src = reinterpret_cast<const uint4*>(q + at * D + q_part * 64);
+    out = quad_rows(o, b, h, n_q, heads, D, row);
+    q_rows = quad_rows(q, b, h, n_q, heads, D, row);
   }
-  __device__ void load_q(uint32_t (&qr)[32]) const {
+  // elements [64 q_part, 64 q_part + 64) of the lane's own Q row, as the 32 packed words tensor memory takes
+  __device__ void load_q(uint32_t (&qr)[32], int q_part, int lane) const {
 #pragma unroll
-    for (int v = 0; v < 8; ++v) {
-      const uint4 t = in_range ? q_src[v] : make_uint4(0, 0, 0, 0);
-      qr[4 * v] = t.x; qr[4 * v + 1] = t.y; qr[4 * v + 2] = t.z; qr[4 * v + 3] = t.w;
+    for (int half = 0; half < 2; ++half) {
+      uint4 ch[4];
+      load_quad_rows(ch, q_rows, q_part * 64 + half * 32, lane);
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        qr[16 * half + 4 * v] = ch[v].x; qr[16 * half + 4 * v + 1] = ch[v].y;
+        qr[16 * half + 4 * v + 2] = ch[v].z; qr[16 * half + 4 * v + 3] = ch[v].w;
+      }
     }
+  }
+  // elements [64 q_part, 64 q_part + 64) of the lane's own Q row, or nullptr if the row does not exist
+  __device__ const uint4* own_q(int q_part, int lane) const {
+    const int j = lane & 3;
+    return j < q_rows.valid ? reinterpret_cast<const uint4*>(q_rows.first + j * q_rows.stride + q_part * 64) : nullptr;
   }
 };
 
@@ -490,6 +545,11 @@ struct FwdTileCtx {
   uint64_t *sdone, *ready;
   volatile int* abort_flag;
   float* mslot;   // [groups][128] floats for the exchange of the first tile's row maxima
+  // the next unit's Q rows, staged 16 bytes per tile: this thread's part of its row (nullptr: the row does not
+  // exist, zeros are staged), the tensor-memory address of that part, and the barrier that collects the parts
+  const uint4* q_next;
+  uint32_t q_next_tmem;
+  uint64_t* q_next_full;
 };
 
 // One key tile J of the CTA's stream; `valid` = valid keys of this group's share (may be <= 0).  Full tiles pass the
@@ -534,6 +594,39 @@ __device__ __forceinline__ void fwd_fast_tile(const FwdTileCtx& c, int J, int va
   mbar_arrive(c.ready + J % 4);
 }
 
+// A run of `count` full key tiles that do not open a unit, from tile J of the stream on: the loop in which the
+// kernel spends its time.  Compiled out of line and handed plain values only (shared-memory addresses as 32-bit
+// numbers), so that its code does not depend on what the bookkeeping between units needs around it.  kQ: each tile
+// also carries one 16-byte chunk (kq, kq + 1, ...) of the thread's part of the next unit's Q row into tensor memory
+// (q_next == nullptr: the row does not exist, zeros go in); the last chunk (7) is followed by the arrival on
+// q_full.  Returns the row sum.
+template <bool kQ>
+__device__ __noinline__ float fwd_fast_run(uint32_t tmem_lane_g, uint32_t sdone, uint32_t ready, uint32_t abort_flag,
+                                           float scale_log2, float neg_m, float l_run, int J, int count,
+                                           const uint4* q_next, uint32_t q_tmem, uint32_t q_full, int kq) {
+  static_assert(kPolyOf8 == 0, "the out-of-line loop leaves the polynomial's range check out");
+  static_assert(kFwdCols == 32, "one 32-column load per thread and tile");
+  float poly_max = -INFINITY;
+  for (int i = 0; i < count; ++i, ++J) {
+    const uint32_t colS = tmem_lane_g + kFwdColS + (J % kFwdSBufs) * 128;
+    uint4 q_chunk = make_uint4(0, 0, 0, 0);
+    if (kQ && q_next != nullptr) q_chunk = q_next[kq + i];
+    mbar_wait_at(sdone + 8 * (J % 4), (J / 4) & 1, abort_flag);
+    tc_fence_after_sync();
+    uint32_t sv[32], pk[16];
+    tmem_ld32(colS, sv);
+    tmem_wait_ld();
+    l_run += fwd_exp32(sv, 32, scale_log2, neg_m, pk, poly_max);
+    tmem_st16(colS, pk);   // in place: this thread has read all of its S columns
+    if (kQ) tmem_st4(q_tmem + 4 * (kq + i), q_chunk);
+    tmem_wait_st();
+    tc_fence_before_sync();
+    mbar_arrive_at(ready + 8 * (J % 4));
+    if (kQ && kq + i == 7) mbar_arrive_at(q_full);
+  }
+  return l_run;
+}
+
 // Walks the CTA's units.  The epilogue of a unit (O out of tensor memory, normalised, stored) comes after the first
 // key tile of the NEXT unit, whose S was issued two tiles earlier: the P V of that tile is the only thing that has
 // to wait for the epilogue's reads.  The Q rows of the next unit go into the other Q buffer once the first tile of
@@ -552,53 +645,91 @@ __device__ __forceinline__ void fwd_softmax_fast(const FwdUnit<D>& u, const FwdS
   c.scale_log2 = scale_log2;
   c.sdone = bar.sdone; c.ready = bar.ready;
   c.abort_flag = u.abort_flag;
-  // the epilogue of the unit before (unit `unit`, the CTA's n-th), whose reference, row sum and verdict are kept
+  // the epilogue of the unit before (at position `pos`, the CTA's n-th), whose reference, row sum and verdict are kept
   float m_prev = 0.f, l_prev = 0.f;
   bool ok_prev = true;
-  auto finish = [&](int unit, int n) {
-    const FwdRow<D> row(sch, unit, r, g, q, n_q, heads, o, lse);
+  auto finish = [&](const FwdPos& pos, int n) {
+    const FwdRow<D> row(sch, pos, r, q, n_q, heads, o, lse);
     float* ex = u.smax + (n & 1) * kFwdGroups * kTile;   // alternates: a fast thread may be a unit ahead
     const bool fin = fwd_epilogue<D>(u, bar.o_full, n & 1, bar.o_free, ex, g, r, c.tmem_lane, m_prev, l_prev,
-                                     row.in_range, row.dst, row.lse_dst);
+                                     row.out, row.in_range, row.lse_dst);
     if (!(fin && ok_prev)) atomicOr(redo_bits + (n >> 5), 1u << (n & 31));
   };
   const int c0 = segs.count[0], T = u.n_tiles;
+  const uint32_t lane_g = c.tmem_lane + g * kFwdCols;
+  const uint32_t sdone_at = smem_u32(bar.sdone), ready_at = smem_u32(bar.ready);
+  const uint32_t abort_at = smem_u32(const_cast<int*>(u.abort_flag));
+  // With enough tiles in a unit the next unit's Q rows travel with tiles 1..8; else in one piece after tile 0.
+  const bool spread = T >= 11;
+  FwdPos pos(sch, sch.first);
   int n = 0;
   for (int unit = sch.first; unit < sch.total; unit += sch.stride, ++n) {
     const bool has_next = unit + sch.stride < sch.total;
     const int J = n * T;
     float m_ref = 0.f, l_run = 0.f, poly_max = -INFINITY;
     c.mslot = u.smax + (2 + (n & 1)) * kFwdGroups * kTile;   // alternates for the same reason
-    // where the next unit's Q rows are: worked out and asked for (into L2) now, fetched after the first tile
-    const FwdRow<D> next_row(sch, has_next ? unit + sch.stride : unit, r, g, q, n_q, heads, o, lse);
-    if (has_next && stages_q && next_row.in_range) prefetch_l2(next_row.q_src);
     if (c0 >= kTile) fwd_fast_tile<true>(c, J, kFwdCols, m_ref, l_run, poly_max);
     else fwd_fast_tile<true>(c, J, c0 - kFwdCols * g, m_ref, l_run, poly_max);
-    if (n > 0) finish(unit - sch.stride, n - 1);
-    if (has_next && stages_q) {
-      uint32_t qr[32];
-      next_row.load_q(qr);
-      tmem_st32(c.tmem_lane + kFwdColQ + ((n + 1) & 1) * kFwdQCols + g * 32, qr);
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(bar.q_full + ((n + 1) & 1));
+    if (n > 0) {
+      FwdPos prev = pos;
+      prev.back(sch);
+      finish(prev, n - 1);
     }
-    // the other tiles: key ranges one after the other, their full tiles in a loop of their own, then the ragged
-    // last tile if any
+    int kq = 8;   // chunks of the next unit's Q that are in tensor memory (8: nothing to do)
+    if (has_next && stages_q) {
+      FwdPos next = pos;
+      next.forward(sch);
+      const FwdRow<D> next_row(sch, next, r, q, n_q, heads, o, lse);
+      const uint32_t q_tmem = c.tmem_lane + kFwdColQ + ((n + 1) & 1) * kFwdQCols + g * 32;
+      if (spread) {
+        c.q_next = next_row.own_q(g, r & 31);
+        if (c.q_next != nullptr) prefetch_l2(c.q_next);   // 128 bytes = one line; asked for now, fetched from tile 1 on
+        c.q_next_tmem = q_tmem;
+        c.q_next_full = bar.q_full + ((n + 1) & 1);
+        kq = 0;
+      } else {
+        uint32_t qr[32];
+        next_row.load_q(qr, g, r & 31);
+        tmem_st32(q_tmem, qr);
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(bar.q_full + ((n + 1) & 1));
+      }
+    }
+    // the other tiles: key ranges one after the other, their full tiles in loops of their own (first those that
+    // carry a piece of Q), then the ragged last tile if any
     int Jr = J + 1;
     for (int sg = 0; sg < segs.n; ++sg) {
       int full = segs.count[sg] / kTile, rest = segs.count[sg] % kTile;
       if (sg == 0) {   // minus the first tile
         if (full > 0) --full; else rest = 0;
       }
-      for (int t = 0; t < full; ++t, ++Jr) fwd_fast_tile<false>(c, Jr, kFwdCols, m_ref, l_run, poly_max);
+      if (full > 0 && kq < 8) {   // full tiles that carry a piece of Q
+        const int cnt = full < 8 - kq ? full : 8 - kq;
+        l_run = fwd_fast_run<true>(lane_g, sdone_at, ready_at, abort_at, scale_log2, -m_ref, l_run, Jr, cnt, c.q_next,
+                                   c.q_next_tmem, smem_u32(c.q_next_full), kq);
+        Jr += cnt; kq += cnt; full -= cnt;
+      }
+      if (full > 0) {
+        l_run = fwd_fast_run<false>(lane_g, sdone_at, ready_at, abort_at, scale_log2, -m_ref, l_run, Jr, full, nullptr,
+                                    0, 0, 0);
+        Jr += full;
+      }
       if (rest) { fwd_fast_tile<false>(c, Jr, rest - kFwdCols * g, m_ref, l_run, poly_max); ++Jr; }
+    }
+    if (kq < 8) {   // the unit had fewer than 8 full tiles after its first: the rest of Q in one go
+      for (; kq < 8; ++kq) tmem_st4(c.q_next_tmem + 4 * kq, c.q_next != nullptr ? c.q_next[kq] : make_uint4(0, 0, 0, 0));
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(c.q_next_full);
     }
     ok_prev = (l_run < kFastSumLimit) && !(poly_max > kPolyArgLimit);   // false for inf and NaN too
     m_prev = m_ref;
     l_prev = l_run;
+    pos.forward(sch);
   }
-  finish(sch.first + (n - 1) * sch.stride, n - 1);
+  pos.back(sch);
+  finish(pos, n - 1);
 }
 
 // ---------------------------------------------------------------------------------- softmax, safe pass
@@ -610,7 +741,7 @@ __device__ __forceinline__ void fwd_softmax_fast(const FwdUnit<D>& u, const FwdS
 // decision) to take the tile's true maximum as the new reference, rescaling O and the row sums.
 template <int D>
 __device__ __forceinline__ void fwd_softmax_safe(const FwdUnit<D>& u, const FwdBars& bar, int warp, int r,
-                                                 float scale_log2, bool in_range, __nv_bfloat16* dst,
+                                                 float scale_log2, const QuadRows& out, bool in_range,
                                                  float* lse_dst) {
   const KeySegs& segs = *u.segs;
   const int g = warp >> 2;
@@ -708,21 +839,21 @@ __device__ __forceinline__ void fwd_softmax_safe(const FwdUnit<D>& u, const FwdB
     tc_fence_before_sync();
     mbar_arrive(bar.p_full + g * kFwdSBufs + buf);
   }
-  fwd_epilogue<D>(u, bar.o_full, 0, nullptr, u.smax, g, r, tmem_lane, m_run, l_run, in_range, dst, lse_dst);
+  fwd_epilogue<D>(u, bar.o_full, 0, nullptr, u.smax, g, r, tmem_lane, m_run, l_run, out, in_range, lse_dst);
 }
 
 // The safe pass of one unit, all roles.  Kept out of line: it is the rare path, and the registers it needs must not
 // weigh on the allocation of the fast pass around it.
 template <int D>
 __device__ __noinline__ void fwd_safe_unit(const FwdUnit<D>& u, const FwdBars& bar, int warp, int lane, int r,
-                                           float scale_log2, bool in_range, __nv_bfloat16* dst, float* lse_dst) {
+                                           float scale_log2, const QuadRows& out, bool in_range, float* lse_dst) {
   constexpr int kMmaWarp = 4 * kFwdGroups, kTmaWarp = 4 * kFwdGroups + 1;
   if (warp == kTmaWarp) {
     if (lane == 0) fwd_produce<D>(u, bar);
   } else if (warp == kMmaWarp) {
     if (lane == 0) fwd_issue<D>(u, bar);
   } else {
-    fwd_softmax_safe<D>(u, bar, warp, r, scale_log2, in_range, dst, lse_dst);
+    fwd_softmax_safe<D>(u, bar, warp, r, scale_log2, out, in_range, lse_dst);
   }
 }
 
@@ -762,7 +893,7 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   const int r = tid & 127;           // query row inside the tile = TMEM lane (softmax warps)
   const bool stages_q = warp < kMmaWarp && (warp >> 2) < D / 64;
   uint32_t qr[32];
-  if (stages_q && !force_safe) FwdRow<D>(sch, sch.first, r, warp >> 2, q, n_q, heads, o, lse).load_q(qr);
+  if (stages_q && !force_safe) FwdRow<D>(sch, sch.first, r, q, n_q, heads, o, lse).load_q(qr, warp >> 2, lane);
   if (warp == kTmaWarp && lane == 0) {
     tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc); tma_prefetch_desc(&tm_kx); tma_prefetch_desc(&tm_vx0);
   }
@@ -824,13 +955,13 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
     int qt;
     sch.decode(unit, qt, u.h, u.b);
     u.bx = cache_shared ? 0 : u.b;
-    const FwdRow<D> row(sch, unit, r, warp >> 2, q, n_q, heads, o, lse);
+    const FwdRow<D> row(sch, unit, r, q, n_q, heads, o, lse);
     if (tid == 0) {
       bar_safe.rearm(1, 128);
       fence_mbar_init();
     }
     if (stages_q) {
-      row.load_q(qr);
+      row.load_q(qr, warp >> 2, lane);
       tmem_st32(tmem_lane + kFwdColQ + (warp >> 2) * 32, qr);
       tmem_wait_st();
     }
@@ -838,7 +969,7 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
     __syncthreads();
     tc_fence_after_sync();
     const FwdUnit<D> su = u;   // a copy: `u` itself never leaves the registers of the fast pass
-    fwd_safe_unit<D>(su, bar_safe, warp, lane, r, scale_log2, row.in_range, row.dst, row.lse_dst);
+    fwd_safe_unit<D>(su, bar_safe, warp, lane, r, scale_log2, row.out, row.in_range, row.lse_dst);
   }
   settle_after_abort(abort_flag);
   tc_fence_before_sync();

@@ -243,9 +243,9 @@ chunk_attn_fwd_pair_kernel(const __nv_bfloat16* __restrict__ q, const __grid_con
     FwdUnit<D> u;
     u.smax = smax;
     u.abort_flag = abort_flag;
-    __nv_bfloat16* dst = o + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D;
+    const QuadRows out = quad_rows(o, b, h, n_q, heads, D, row);
     float* lse_dst = lse ? lse + (static_cast<size_t>(b) * heads + h) * n_q + (in_range ? row : 0) : nullptr;
-    ok = fwd_epilogue<D, kPairGroups>(u, bar.o_full, 0, nullptr, u.smax, g, r, tmem_lane, m_ref, l_run, in_range, dst, lse_dst) && ok;
+    ok = fwd_epilogue<D, kPairGroups>(u, bar.o_full, 0, nullptr, u.smax, g, r, tmem_lane, m_ref, l_run, out, in_range, lse_dst) && ok;
     if (!ok) *needs_safe = 1;
   }
 

@@ -94,6 +94,46 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return ok;
 }
 
+// The same waits and arrivals on 32-bit shared-memory addresses (of the barrier and of the abort flag): for code
+// that is compiled out of line, where a generic pointer would have to be converted at every use.
+__device__ __forceinline__ bool mbar_try_wait_at(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void mbar_arrive_at(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_at(uint32_t bar, uint32_t parity, uint32_t abort_flag) {
+  bool ok = mbar_try_wait_at(bar, parity);
+  if (!ok) {
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    while (!(ok = mbar_try_wait_at(bar, parity))) {
+      if ((++it & 63u) == 0) {
+        uint32_t aborted;
+        asm volatile("ld.volatile.shared::cta.u32 %0, [%1];" : "=r"(aborted) : "r"(abort_flag) : "memory");
+        if (aborted) break;
+        if (clock64() - t0 > kWaitCycleLimit) {
+          asm volatile("st.volatile.shared::cta.u32 [%0], %1;" ::"r"(abort_flag), "r"(1u) : "memory");
+          atomicOr(&g_device_status, kStatusWaitTimeout);
+          break;
+        }
+      }
+    }
+  }
+  __syncwarp();
+  return ok;
+}
+
 // Barrier among `threads` threads of the CTA (a multiple of 32) that all name the same id (1..15).
 __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
@@ -228,6 +268,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
       "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
       "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
+}
+__device__ __forceinline__ void tmem_st4(uint32_t taddr, const uint4& r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};" ::"r"(taddr), "r"(r.x), "r"(r.y),
+               "r"(r.z), "r"(r.w)
+               : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
