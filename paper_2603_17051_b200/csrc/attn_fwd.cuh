@@ -3,7 +3,8 @@
 // Warp-specialised, one CTA per SM:
 //   four softmax groups of 4 warps: group g owns keys [32 g, 32 g + 32) of every key tile, one query row
 //   per thread (four warps per scheduler: while one waits for tensor memory or a barrier the others keep the
-//   special-function unit busy); then one warp whose first thread issues every tcgen05 MMA, one for TMA loads
+//   special-function unit busy); then one warp whose first thread issues every tcgen05 MMA, one for TMA loads, and
+//   four epilogue warps that write O and LSE out and bring the next units' Q rows in (fast pass)
 // Q lives in tensor memory (bf16 pairs, written once by the softmax threads) and is the A operand of
 // S = Q K^T, so shared memory only carries K and V: an MMA with both operands in shared memory reads
 // 128 B/clk, the whole shared-memory bandwidth, and then competes with the TMA writes of the next tiles.
@@ -35,15 +36,16 @@ namespace astro {
 constexpr int kFwdKStages = 3, kFwdVStages = 3, kFwdSBufs = 2;
 constexpr int kFwdGroups = 4;                    // layer shape, forward alone: 2 groups 0.741 ms, 4 groups 0.713 ms
 constexpr int kFwdCols = kTile / kFwdGroups;     // keys per group and tile
-constexpr int kFwdThreads = 128 * kFwdGroups + 64;
+constexpr int kFwdEpiWarps = 4;                    // fast pass: warps that write O and LSE out and stage Q
+constexpr int kFwdThreads = 128 * kFwdGroups + 64 + 32 * kFwdEpiWarps;
 constexpr int kFwdBarSlots = 32;                 // mbarriers of one pass
 constexpr int kFwdMaxUnits = 1024;               // work units one CTA may walk (one redo bit each)
 
 template <int D> struct FwdSmem {
   static constexpr int kK = 0;
   static constexpr int kV = kK + kFwdKStages * TileGeom<D>::kBytes;
-  static constexpr int kMax = kV + kFwdVStages * TileGeom<D>::kBytes;  // float [4][groups][128]: exchange slots
-  static constexpr int kBars = kMax + 4 * kFwdGroups * kTile * 4;      // two sets of barriers, 3 words, redo bits
+  static constexpr int kMax = kV + kFwdVStages * TileGeom<D>::kBytes;  // float [4][groups][128] + [2][128]: exchange slots
+  static constexpr int kBars = kMax + (4 * kFwdGroups + 2) * kTile * 4;  // two sets of barriers, 3 words, redo bits
   static constexpr int kTotal = kBars + 2 * kFwdBarSlots * 8 + 64 + kFwdMaxUnits / 8 + 1024;  // + slack to align to 1024
 };
 
@@ -209,19 +211,22 @@ struct FwdCursor {
 // byte count plus the TMA completions) and the arrival of every softmax thread that has stored its P(J).
 // sdone[J % 4] is committed behind S(J): S(J) is ready for the softmax threads, and -- MMAs complete in order --
 // the P V of tile J-2 is done too, so the producer may refill the K stage of tile J and the V stage of tile J-2.
-// Per unit: q_full[n % 2] (the unit's Q rows are in tensor memory buffer n % 2), o_full (its last P V is done),
-// o_free (every softmax thread has read its part of O: the next unit's first P V may overwrite it).
+// Per unit: q_full[n % 2] (the unit's Q rows are in tensor memory buffer n % 2), stats_full[n % 2] (every softmax
+// thread has left its row sum, and the row's reference, in shared memory), o_full (the unit's last P V is done),
+// o_free (the epilogue warps have read O out of tensor memory: the next unit's first P V may overwrite it).
 struct FwdFastBars {
-  uint64_t *q_full, *k01, *ready, *sdone, *o_full, *o_free;
+  uint64_t *q_full, *k01, *ready, *sdone, *o_full, *o_free, *stats_full;
   __device__ explicit FwdFastBars(uint64_t* b)
-      : q_full(b), k01(b + 2), ready(b + 3), sdone(b + 7), o_full(b + 11), o_free(b + 12) {}
-  __device__ void init(int q_count) const {
-    mbar_init(q_full, q_count);
-    mbar_init(q_full + 1, q_count);
+      : q_full(b), k01(b + 2), ready(b + 3), sdone(b + 7), o_full(b + 11), o_free(b + 12), stats_full(b + 13) {}
+  __device__ void init() const {
+    mbar_init(q_full, 32 * kFwdEpiWarps);
+    mbar_init(q_full + 1, 32 * kFwdEpiWarps);
     mbar_init(k01, 1);
     for (int i = 0; i < 4; ++i) { mbar_init(ready + i, 1 + 128 * kFwdGroups); mbar_init(sdone + i, 1); }
     mbar_init(o_full, 1);
-    mbar_init(o_free, 128 * kFwdGroups);
+    mbar_init(o_free, 32 * kFwdEpiWarps);
+    mbar_init(stats_full, 128 * kFwdGroups);
+    mbar_init(stats_full + 1, 128 * kFwdGroups);
   }
 };
 
@@ -437,7 +442,34 @@ __device__ __forceinline__ float fwd_exp32(const uint32_t (&s)[32], int valid, f
   return r0 + r1;
 }
 
-// Epilogue shared by both passes: row sum = sum of the groups' partial sums; 32-column slices of the output
+// 32 accumulator columns of the lane's row -> times 1/l -> bf16 -> columns [col0, col0 + 32) of the output row, the
+// quads of the warp storing their rows together.  chk2 stays 0 while every value times 0 is 0, i.e. is finite.
+__device__ __forceinline__ void fwd_store_slice(const uint32_t (&acc)[32], uint64_t inv2, uint64_t& chk2,
+                                                const QuadRows& out, int col0, int lane) {
+  const uint64_t zero2 = f32x2(0.f, 0.f);
+  uint4 ch[4];
+#pragma unroll
+  for (int v = 0; v < 4; ++v) {
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint64_t f2 = mul2(f32x2(__uint_as_float(acc[8 * v + 2 * e]), __uint_as_float(acc[8 * v + 2 * e + 1])), inv2);
+      chk2 = fma2(f2, zero2, chk2);
+      float f0, f1;
+      f32x2_split(f2, f0, f1);
+      w[e] = pack_bf16(f0, f1);
+    }
+    ch[v] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  store_quad_rows(ch, out, col0, lane);
+}
+__device__ __forceinline__ bool fwd_all_finite(uint64_t chk2) {
+  float chk0, chk1;
+  f32x2_split(chk2, chk0, chk1);
+  return chk0 == 0.f && chk1 == 0.f;
+}
+
+// Epilogue shared by the safe pass and the CTA-pair kernel: row sum = sum of the groups' partial sums; 32-column slices of the output
 // row are dealt round-robin to the groups.  The slices are read out of tensor memory first; `o_free`, if given,
 // gets this thread's arrival right after that (O may be overwritten from then on).  `ex` = [G][128] floats for the
 // exchange of the partial sums.  The quads of a warp store their rows together (64 contiguous bytes per row).
@@ -465,32 +497,16 @@ __device__ __forceinline__ bool fwd_epilogue(const FwdUnit<D>& u, uint64_t* o_fu
 #pragma unroll
   for (int og = 0; og < G; ++og) l += ex[og * kTile + r];
   const float inv_l = 1.f / l;
-  const uint64_t inv2 = f32x2(inv_l, inv_l), zero2 = f32x2(0.f, 0.f);
-  uint64_t chk2 = zero2;   // stays 0 while every value times 0 is 0, i.e. while every value is finite
+  const uint64_t inv2 = f32x2(inv_l, inv_l);
+  uint64_t chk2 = f32x2(0.f, 0.f);
 #pragma unroll
   for (int i = 0; i < kOwn; ++i) {
     const int c4 = g + i * G;
     if (c4 >= kSlices) continue;   // the same for the whole warp
-    uint4 ch[4];
-#pragma unroll
-    for (int v = 0; v < 4; ++v) {
-      uint32_t w[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const uint64_t f2 = mul2(f32x2(__uint_as_float(acc[i][8 * v + 2 * e]), __uint_as_float(acc[i][8 * v + 2 * e + 1])), inv2);
-        chk2 = fma2(f2, zero2, chk2);
-        float f0, f1;
-        f32x2_split(f2, f0, f1);
-        w[e] = pack_bf16(f0, f1);
-      }
-      ch[v] = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-    store_quad_rows(ch, out, c4 * 32, r & 31);
+    fwd_store_slice(acc[i], inv2, chk2, out, c4 * 32, r & 31);
   }
   if (g == G - 1 && in_range && lse_dst != nullptr) *lse_dst = (m_run + log2f(l)) * 0.6931471805599453f;
-  float chk0, chk1;
-  f32x2_split(chk2, chk0, chk1);
-  return chk0 == 0.f && chk1 == 0.f;
+  return fwd_all_finite(chk2);
 }
 
 // Where the rows of a unit are: the lane's own row for LSE, its quad's rows for O and Q.
@@ -529,11 +545,6 @@ template <int D> struct FwdRow {
       }
     }
   }
-  // elements [64 q_part, 64 q_part + 64) of the lane's own Q row, or nullptr if the row does not exist
-  __device__ const uint4* own_q(int q_part, int lane) const {
-    const int j = lane & 3;
-    return j < q_rows.valid ? reinterpret_cast<const uint4*>(q_rows.first + j * q_rows.stride + q_part * 64) : nullptr;
-  }
 };
 
 // ---------------------------------------------------------------------------------- softmax, fast pass
@@ -545,11 +556,6 @@ struct FwdTileCtx {
   uint64_t *sdone, *ready;
   volatile int* abort_flag;
   float* mslot;   // [groups][128] floats for the exchange of the first tile's row maxima
-  // the next unit's Q rows, staged 16 bytes per tile: this thread's part of its row (nullptr: the row does not
-  // exist, zeros are staged), the tensor-memory address of that part, and the barrier that collects the parts
-  const uint4* q_next;
-  uint32_t q_next_tmem;
-  uint64_t* q_next_full;
 };
 
 // One key tile J of the CTA's stream; `valid` = valid keys of this group's share (may be <= 0).  Full tiles pass the
@@ -596,21 +602,15 @@ __device__ __forceinline__ void fwd_fast_tile(const FwdTileCtx& c, int J, int va
 
 // A run of `count` full key tiles that do not open a unit, from tile J of the stream on: the loop in which the
 // kernel spends its time.  Compiled out of line and handed plain values only (shared-memory addresses as 32-bit
-// numbers), so that its code does not depend on what the bookkeeping between units needs around it.  kQ: each tile
-// also carries one 16-byte chunk (kq, kq + 1, ...) of the thread's part of the next unit's Q row into tensor memory
-// (q_next == nullptr: the row does not exist, zeros go in); the last chunk (7) is followed by the arrival on
-// q_full.  Returns the row sum.
-template <bool kQ>
+// numbers), so that its code does not depend on what the bookkeeping between units needs around it.
+// Returns the row sum.
 __device__ __noinline__ float fwd_fast_run(uint32_t tmem_lane_g, uint32_t sdone, uint32_t ready, uint32_t abort_flag,
-                                           float scale_log2, float neg_m, float l_run, int J, int count,
-                                           const uint4* q_next, uint32_t q_tmem, uint32_t q_full, int kq) {
+                                           float scale_log2, float neg_m, float l_run, int J, int count) {
   static_assert(kPolyOf8 == 0, "the out-of-line loop leaves the polynomial's range check out");
   static_assert(kFwdCols == 32, "one 32-column load per thread and tile");
   float poly_max = -INFINITY;
   for (int i = 0; i < count; ++i, ++J) {
     const uint32_t colS = tmem_lane_g + kFwdColS + (J % kFwdSBufs) * 128;
-    uint4 q_chunk = make_uint4(0, 0, 0, 0);
-    if (kQ && q_next != nullptr) q_chunk = q_next[kq + i];
     mbar_wait_at(sdone + 8 * (J % 4), (J / 4) & 1, abort_flag);
     tc_fence_after_sync();
     uint32_t sv[32], pk[16];
@@ -618,118 +618,143 @@ __device__ __noinline__ float fwd_fast_run(uint32_t tmem_lane_g, uint32_t sdone,
     tmem_wait_ld();
     l_run += fwd_exp32(sv, 32, scale_log2, neg_m, pk, poly_max);
     tmem_st16(colS, pk);   // in place: this thread has read all of its S columns
-    if (kQ) tmem_st4(q_tmem + 4 * (kq + i), q_chunk);
     tmem_wait_st();
     tc_fence_before_sync();
     mbar_arrive_at(ready + 8 * (J % 4));
-    if (kQ && kq + i == 7) mbar_arrive_at(q_full);
   }
   return l_run;
 }
 
-// Walks the CTA's units.  The epilogue of a unit (O out of tensor memory, normalised, stored) comes after the first
-// key tile of the NEXT unit, whose S was issued two tiles earlier: the P V of that tile is the only thing that has
-// to wait for the epilogue's reads.  The Q rows of the next unit go into the other Q buffer once the first tile of
-// the current unit is through (every S of the unit before, the buffer's last reader, is complete by then).
+// Where the fast pass leaves a unit's row statistics for the epilogue warps: per unit parity, the groups' partial
+// row sums [groups][128] and the rows' reference exponents [128].
+template <int D> struct FwdStats {
+  float* smax;
+  __device__ float* sums(int n) const { return smax + (n & 1) * kFwdGroups * kTile; }
+  __device__ float* refs(int n) const { return smax + 4 * kFwdGroups * kTile + (n & 1) * kTile; }
+  __device__ float* maxima(int n) const { return smax + (2 + (n & 1)) * kFwdGroups * kTile; }   // first-tile exchange
+};
+
+// Walks the CTA's units: per unit the first key tile (which fixes the rows' reference), the others, then the row
+// sum and the reference go to shared memory for the epilogue warps.  Nothing else happens between the last tile of a
+// unit and the first of the next, whose S was issued two tiles earlier.
 // A unit one of whose rows must be redone by the safe pass gets its bit set in `redo_bits`.
 template <int D>
 __device__ __forceinline__ void fwd_softmax_fast(const FwdUnit<D>& u, const FwdSched& sch, const FwdFastBars& bar,
-                                                 int warp, int r, float scale_log2, const __nv_bfloat16* q, int n_q,
-                                                 int heads, __nv_bfloat16* o, float* lse, uint32_t* redo_bits) {
+                                                 int warp, int r, float scale_log2, uint32_t* redo_bits) {
   const KeySegs& segs = *u.segs;
   const int g = warp >> 2;
-  const bool stages_q = g < D / 64;
+  const FwdStats<D> stats{u.smax};
   FwdTileCtx c;
   c.tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
   c.g = g; c.r = r; c.warp = warp;
   c.scale_log2 = scale_log2;
   c.sdone = bar.sdone; c.ready = bar.ready;
   c.abort_flag = u.abort_flag;
-  // the epilogue of the unit before (at position `pos`, the CTA's n-th), whose reference, row sum and verdict are kept
-  float m_prev = 0.f, l_prev = 0.f;
-  bool ok_prev = true;
-  auto finish = [&](const FwdPos& pos, int n) {
-    const FwdRow<D> row(sch, pos, r, q, n_q, heads, o, lse);
-    float* ex = u.smax + (n & 1) * kFwdGroups * kTile;   // alternates: a fast thread may be a unit ahead
-    const bool fin = fwd_epilogue<D>(u, bar.o_full, n & 1, bar.o_free, ex, g, r, c.tmem_lane, m_prev, l_prev,
-                                     row.out, row.in_range, row.lse_dst);
-    if (!(fin && ok_prev)) atomicOr(redo_bits + (n >> 5), 1u << (n & 31));
-  };
   const int c0 = segs.count[0], T = u.n_tiles;
   const uint32_t lane_g = c.tmem_lane + g * kFwdCols;
   const uint32_t sdone_at = smem_u32(bar.sdone), ready_at = smem_u32(bar.ready);
   const uint32_t abort_at = smem_u32(const_cast<int*>(u.abort_flag));
-  // With enough tiles in a unit the next unit's Q rows travel with tiles 1..8; else in one piece after tile 0.
-  const bool spread = T >= 11;
-  FwdPos pos(sch, sch.first);
   int n = 0;
   for (int unit = sch.first; unit < sch.total; unit += sch.stride, ++n) {
-    const bool has_next = unit + sch.stride < sch.total;
     const int J = n * T;
     float m_ref = 0.f, l_run = 0.f, poly_max = -INFINITY;
-    c.mslot = u.smax + (2 + (n & 1)) * kFwdGroups * kTile;   // alternates for the same reason
+    c.mslot = stats.maxima(n);   // alternates: a fast thread may be a unit ahead of the others
     if (c0 >= kTile) fwd_fast_tile<true>(c, J, kFwdCols, m_ref, l_run, poly_max);
     else fwd_fast_tile<true>(c, J, c0 - kFwdCols * g, m_ref, l_run, poly_max);
-    if (n > 0) {
-      FwdPos prev = pos;
-      prev.back(sch);
-      finish(prev, n - 1);
-    }
-    int kq = 8;   // chunks of the next unit's Q that are in tensor memory (8: nothing to do)
-    if (has_next && stages_q) {
-      FwdPos next = pos;
-      next.forward(sch);
-      const FwdRow<D> next_row(sch, next, r, q, n_q, heads, o, lse);
-      const uint32_t q_tmem = c.tmem_lane + kFwdColQ + ((n + 1) & 1) * kFwdQCols + g * 32;
-      if (spread) {
-        c.q_next = next_row.own_q(g, r & 31);
-        if (c.q_next != nullptr) prefetch_l2(c.q_next);   // 128 bytes = one line; asked for now, fetched from tile 1 on
-        c.q_next_tmem = q_tmem;
-        c.q_next_full = bar.q_full + ((n + 1) & 1);
-        kq = 0;
-      } else {
-        uint32_t qr[32];
-        next_row.load_q(qr, g, r & 31);
-        tmem_st32(q_tmem, qr);
-        tmem_wait_st();
-        tc_fence_before_sync();
-        mbar_arrive(bar.q_full + ((n + 1) & 1));
-      }
-    }
-    // the other tiles: key ranges one after the other, their full tiles in loops of their own (first those that
-    // carry a piece of Q), then the ragged last tile if any
+    // the other tiles: key ranges one after the other, their full tiles in one run, then the ragged last tile if any
     int Jr = J + 1;
     for (int sg = 0; sg < segs.n; ++sg) {
       int full = segs.count[sg] / kTile, rest = segs.count[sg] % kTile;
       if (sg == 0) {   // minus the first tile
         if (full > 0) --full; else rest = 0;
       }
-      if (full > 0 && kq < 8) {   // full tiles that carry a piece of Q
-        const int cnt = full < 8 - kq ? full : 8 - kq;
-        l_run = fwd_fast_run<true>(lane_g, sdone_at, ready_at, abort_at, scale_log2, -m_ref, l_run, Jr, cnt, c.q_next,
-                                   c.q_next_tmem, smem_u32(c.q_next_full), kq);
-        Jr += cnt; kq += cnt; full -= cnt;
-      }
       if (full > 0) {
-        l_run = fwd_fast_run<false>(lane_g, sdone_at, ready_at, abort_at, scale_log2, -m_ref, l_run, Jr, full, nullptr,
-                                    0, 0, 0);
+        l_run = fwd_fast_run(lane_g, sdone_at, ready_at, abort_at, scale_log2, -m_ref, l_run, Jr, full);
         Jr += full;
       }
       if (rest) { fwd_fast_tile<false>(c, Jr, rest - kFwdCols * g, m_ref, l_run, poly_max); ++Jr; }
     }
-    if (kq < 8) {   // the unit had fewer than 8 full tiles after its first: the rest of Q in one go
-      for (; kq < 8; ++kq) tmem_st4(c.q_next_tmem + 4 * kq, c.q_next != nullptr ? c.q_next[kq] : make_uint4(0, 0, 0, 0));
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(c.q_next_full);
+    // The slots of unit n - 2 are free: the epilogue warps read them before they let go of that unit's O, which the
+    // first P V of unit n - 1 waited for.
+    stats.sums(n)[g * kTile + r] = l_run;
+    if (g == 0) stats.refs(n)[r] = m_ref;
+    if (!((l_run < kFastSumLimit) && !(poly_max > kPolyArgLimit)))   // true for inf and NaN too
+      atomicOr(redo_bits + (n >> 5), 1u << (n & 31));
+    mbar_arrive(bar.stats_full + (n & 1));
+  }
+}
+
+// ---------------------------------------------------------------------------------- epilogue warps, fast pass
+// Four warps (one per quarter of the tensor-memory lanes; lane = query row of the tile).  Per unit: wait for the row
+// statistics and for the last P V, read O out of tensor memory (two 32-column slices at a time; o_free after the last
+// read), normalise, store O and LSE; then fetch the Q rows of the unit after the next into the Q buffer this unit used.
+// They keep every load from and store to global memory away from the softmax threads.
+template <int D>
+__device__ __forceinline__ void fwd_epilogue_fast(const FwdUnit<D>& u, const FwdSched& sch, const FwdFastBars& bar,
+                                                  int warp, int lane, const __nv_bfloat16* q, int n_q, int heads,
+                                                  __nv_bfloat16* o, float* lse, uint32_t* redo_bits) {
+  constexpr int kSlices = D / 32;
+  const FwdStats<D> stats{u.smax};
+  const int r = (warp & 3) * 32 + lane;
+  const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+  auto stage_q = [&](const FwdPos& pos, int buf) {
+    const FwdRow<D> row(sch, pos, r, q, n_q, heads, o, lse);
+#pragma unroll
+    for (int part = 0; part < D / 64; ++part) {
+      uint32_t qr[32];
+      row.load_q(qr, part, lane);
+      tmem_st32(tmem_lane + kFwdColQ + buf * kFwdQCols + part * 32, qr);
     }
-    ok_prev = (l_run < kFastSumLimit) && !(poly_max > kPolyArgLimit);   // false for inf and NaN too
-    m_prev = m_ref;
-    l_prev = l_run;
+    tmem_wait_st();
+    tc_fence_before_sync();
+    mbar_arrive(bar.q_full + buf);
+  };
+  FwdPos pos(sch, sch.first);
+  {   // the first two units' Q
+    stage_q(pos, 0);
+    if (sch.first + sch.stride < sch.total) {
+      FwdPos next = pos;
+      next.forward(sch);
+      stage_q(next, 1);
+    }
+  }
+  int n = 0;
+  for (int unit = sch.first; unit < sch.total; unit += sch.stride, ++n) {
+    const FwdRow<D> row(sch, pos, r, q, n_q, heads, o, lse);
+    mbar_wait_relaxed(bar.stats_full + (n & 1), (n >> 1) & 1, u.abort_flag);
+    float l = 0.f;
+#pragma unroll
+    for (int g = 0; g < kFwdGroups; ++g) l += stats.sums(n)[g * kTile + r];
+    const float m = stats.refs(n)[r];
+    const float inv_l = 1.f / l;
+    const uint64_t inv2 = f32x2(inv_l, inv_l);
+    uint64_t chk2 = f32x2(0.f, 0.f);
+    mbar_wait(bar.o_full, n & 1, u.abort_flag);
+    tc_fence_after_sync();
+#pragma unroll
+    for (int c4 = 0; c4 < kSlices; c4 += 2) {
+      uint32_t acc[2][32];
+      tmem_ld32(tmem_lane + kFwdColO + c4 * 32, acc[0]);
+      tmem_ld32(tmem_lane + kFwdColO + (c4 + 1) * 32, acc[1]);
+      tmem_wait_ld();
+      if (c4 + 2 >= kSlices) {   // O is in registers (or stored): the next unit may start on it
+        tc_fence_before_sync();
+        mbar_arrive(bar.o_free);
+      }
+      fwd_store_slice(acc[0], inv2, chk2, row.out, c4 * 32, lane);
+      fwd_store_slice(acc[1], inv2, chk2, row.out, (c4 + 1) * 32, lane);
+    }
+    if (row.in_range && row.lse_dst != nullptr) *row.lse_dst = (m + log2f(l)) * 0.6931471805599453f;
+    if (!fwd_all_finite(chk2)) atomicOr(redo_bits + (n >> 5), 1u << (n & 31));
+    // Q of the unit after the next, into this unit's buffer: every S of this unit is complete (o_full)
+    if (unit + 2 * sch.stride < sch.total) {
+      FwdPos later = pos;
+      later.forward(sch);
+      later.forward(sch);
+      stage_q(later, n & 1);
+    }
     pos.forward(sch);
   }
-  pos.back(sch);
-  finish(pos, n - 1);
 }
 
 // ---------------------------------------------------------------------------------- softmax, safe pass
@@ -852,7 +877,7 @@ __device__ __noinline__ void fwd_safe_unit(const FwdUnit<D>& u, const FwdBars& b
     if (lane == 0) fwd_produce<D>(u, bar);
   } else if (warp == kMmaWarp) {
     if (lane == 0) fwd_issue<D>(u, bar);
-  } else {
+  } else if (warp < kMmaWarp) {
     fwd_softmax_safe<D>(u, bar, warp, r, scale_log2, out, in_range, lse_dst);
   }
 }
@@ -887,18 +912,13 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
   sch.stride = gridDim.x;
   sch.total = sch.q_tiles * heads * batch;
 
-  // Each softmax thread fetches its share of the first unit's Q row (64 elements: group g takes elements
-  // [64 g, 64 g + 64)) before anything else, so that the load's latency passes behind the barrier set-up and the
-  // tensor-memory allocation.
   const int r = tid & 127;           // query row inside the tile = TMEM lane (softmax warps)
-  const bool stages_q = warp < kMmaWarp && (warp >> 2) < D / 64;
-  uint32_t qr[32];
-  if (stages_q && !force_safe) FwdRow<D>(sch, sch.first, r, q, n_q, heads, o, lse).load_q(qr, warp >> 2, lane);
+  const bool stages_q = warp < kMmaWarp && (warp >> 2) < D / 64;   // safe pass: who writes Q into tensor memory
   if (warp == kTmaWarp && lane == 0) {
     tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc); tma_prefetch_desc(&tm_kx); tma_prefetch_desc(&tm_vx0);
   }
   if (tid == 0) {
-    bar_fast.init(128 * (D / 64));  // q_full: the threads that write Q into tensor memory
+    bar_fast.init();
     bar_safe.init(1, 128);
     *abort_flag = 0;
     fence_mbar_init();
@@ -931,20 +951,15 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
       if (lane == 0) fwd_produce_fast<D>(u, sch, bar_fast);
     } else if (warp == kMmaWarp) {
       if (lane == 0) fwd_issue_fast<D>(u, sch, bar_fast);
+    } else if (warp < kMmaWarp) {
+      fwd_softmax_fast<D>(u, sch, bar_fast, warp, r, scale_log2, redo_bits);
     } else {
-      // Q row of the first unit -> tensor memory buffer 0 (32 packed columns per 64 elements)
-      if (stages_q) {
-        tmem_st32(tmem_lane + kFwdColQ + (warp >> 2) * 32, qr);
-        tmem_wait_st();
-        tc_fence_before_sync();
-        mbar_arrive(bar_fast.q_full);
-      }
-      fwd_softmax_fast<D>(u, sch, bar_fast, warp, r, scale_log2, q, n_q, heads, o, lse, redo_bits);
+      fwd_epilogue_fast<D>(u, sch, bar_fast, warp, lane, q, n_q, heads, o, lse, redo_bits);
     }
   }
 
   // ---- safe pass, unit by unit, for the units one of whose rows asked for it (every MMA of the fast pass has
-  //      finished by now: the softmax threads waited for the last one before their last epilogue)
+  //      finished by now: the epilogue warps waited for the last one)
   int n = 0;
   for (int unit = sch.first; unit < sch.total; unit += sch.stride, ++n) {
     tc_fence_before_sync();
@@ -961,6 +976,7 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
       fence_mbar_init();
     }
     if (stages_q) {
+      uint32_t qr[32];
       row.load_q(qr, warp >> 2, lane);
       tmem_st32(tmem_lane + kFwdColQ + (warp >> 2) * 32, qr);
       tmem_wait_st();

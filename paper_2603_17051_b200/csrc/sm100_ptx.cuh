@@ -94,6 +94,29 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return ok;
 }
 
+// For warps that wait long and are in nobody's way when they wake up a little late: sleeps between the polls, so
+// that the polling does not take issue slots from the warps that compute.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  bool ok = mbar_try_wait(bar, parity);
+  if (!ok) {
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    while (!(ok = mbar_try_wait(bar, parity))) {
+      __nanosleep(64);
+      if ((++it & 63u) == 0) {
+        if (*abort_flag) break;
+        if (clock64() - t0 > kWaitCycleLimit) {
+          *abort_flag = 1;
+          atomicOr(&g_device_status, kStatusWaitTimeout);
+          break;
+        }
+      }
+    }
+  }
+  __syncwarp();
+  return ok;
+}
+
 // The same waits and arrivals on 32-bit shared-memory addresses (of the barrier and of the abort flag): for code
 // that is compiled out of line, where a generic pointer would have to be converted at every use.
 __device__ __forceinline__ bool mbar_try_wait_at(uint32_t bar, uint32_t parity) {
