@@ -308,10 +308,9 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
     // ---- epilogue: groups 0 and 1 write columns [g D/2, (g+1) D/2) of dQ
     mbar_wait(dq_full, 0, abort_flag);
     tc_fence_after_sync();
-    if (g < 2) {
-      __nv_bfloat16* dst = dq + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + g * (D / 2);
-      store_row_from_tmem<D / 2>(tmem_lane + kColdQ + g * (D / 2), scale, dst, in_range);
-    }
+    if (g < 2)
+      store_rows_from_tmem<D / 2>(tmem_lane + kColdQ + g * (D / 2), scale, quad_rows(dq, b, h, n_q, heads, D, row),
+                                  g * (D / 2), tid & 31);
   }
 
   settle_after_abort(abort_flag);
@@ -530,10 +529,10 @@ chunk_attn_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid
     mbar_wait(acc_full, 0, abort_flag);
     tc_fence_after_sync();
     const int krow = k0 + r;
-    const bool in_range = krow < n_kc;
-    const size_t row_off = ((static_cast<size_t>(b) * n_kc + (in_range ? krow : 0)) * heads + h) * D + g * (D / 2);
-    store_row_from_tmem<D / 2>(tmem_lane + kColdK + g * (D / 2), scale, dk + row_off, in_range);
-    store_row_from_tmem<D / 2>(tmem_lane + kColdV + g * (D / 2), 1.f, dv + row_off, in_range);
+    store_rows_from_tmem<D / 2>(tmem_lane + kColdK + g * (D / 2), scale, quad_rows(dk, b, h, n_kc, heads, D, krow),
+                                g * (D / 2), tid & 31);
+    store_rows_from_tmem<D / 2>(tmem_lane + kColdV + g * (D / 2), 1.f, quad_rows(dv, b, h, n_kc, heads, D, krow),
+                                g * (D / 2), tid & 31);
   }
 
   settle_after_abort(abort_flag);

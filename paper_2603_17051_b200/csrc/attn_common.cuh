@@ -155,28 +155,31 @@ __device__ __forceinline__ void zero_tile_rows_from(uint8_t* smem_tile, int firs
   fence_proxy_async_smem();
 }
 
-// Write one row of D fp32 accumulators (TMEM columns [col0, col0+D) of this thread's lane), times
-// `mult`, as bf16 to `dst` (global, 16-byte aligned) when `store` is set.  Warp-collective.
-template <int D>
-__device__ __forceinline__ void store_row_from_tmem(uint32_t taddr_lane_col0, float mult, __nv_bfloat16* dst,
-                                                    bool store) {
+// Write N fp32 accumulators of this thread's row (TMEM columns [taddr, taddr + N) of its lane), times `mult`, as
+// bf16 into columns [col0, col0 + N) of the row; the quads of the warp store their rows together (64 contiguous
+// bytes per row and access).  Warp-collective.
+template <int N>
+__device__ __forceinline__ void store_rows_from_tmem(uint32_t taddr_lane_col0, float mult, const QuadRows& rows,
+                                                     int col0, int lane) {
+  const uint64_t m2 = f32x2(mult, mult);
 #pragma unroll
-  for (int j = 0; j < D / 32; ++j) {
+  for (int j = 0; j < N / 32; ++j) {
     uint32_t r[32];
     tmem_ld32(taddr_lane_col0 + j * 32, r);
     tmem_wait_ld();
-    if (store) {
-      uint4* out = reinterpret_cast<uint4*>(dst + j * 32);
+    uint4 ch[4];
 #pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        uint4 w;
-        w.x = pack_bf16(__uint_as_float(r[8 * v + 0]) * mult, __uint_as_float(r[8 * v + 1]) * mult);
-        w.y = pack_bf16(__uint_as_float(r[8 * v + 2]) * mult, __uint_as_float(r[8 * v + 3]) * mult);
-        w.z = pack_bf16(__uint_as_float(r[8 * v + 4]) * mult, __uint_as_float(r[8 * v + 5]) * mult);
-        w.w = pack_bf16(__uint_as_float(r[8 * v + 6]) * mult, __uint_as_float(r[8 * v + 7]) * mult);
-        out[v] = w;
+    for (int v = 0; v < 4; ++v) {
+      uint32_t w[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float f0, f1;
+        f32x2_split(mul2(f32x2(__uint_as_float(r[8 * v + 2 * e]), __uint_as_float(r[8 * v + 2 * e + 1])), m2), f0, f1);
+        w[e] = pack_bf16(f0, f1);
       }
+      ch[v] = make_uint4(w[0], w[1], w[2], w[3]);
     }
+    store_quad_rows(ch, rows, col0 + j * 32, lane);
   }
 }
 

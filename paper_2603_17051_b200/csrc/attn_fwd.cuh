@@ -4,7 +4,7 @@
 //   four softmax groups of 4 warps: group g owns keys [32 g, 32 g + 32) of every key tile, one query row
 //   per thread (four warps per scheduler: while one waits for tensor memory or a barrier the others keep the
 //   special-function unit busy); then one warp whose first thread issues every tcgen05 MMA, one for TMA loads, and
-//   four epilogue warps that write O and LSE out and bring the next units' Q rows in (fast pass)
+//   eight epilogue warps that write O and LSE out and bring the next units' Q rows in (fast pass)
 // Q lives in tensor memory (bf16 pairs, written once by the softmax threads) and is the A operand of
 // S = Q K^T, so shared memory only carries K and V: an MMA with both operands in shared memory reads
 // 128 B/clk, the whole shared-memory bandwidth, and then competes with the TMA writes of the next tiles.
@@ -36,7 +36,7 @@ namespace astro {
 constexpr int kFwdKStages = 3, kFwdVStages = 3, kFwdSBufs = 2;
 constexpr int kFwdGroups = 4;                    // layer shape, forward alone: 2 groups 0.741 ms, 4 groups 0.713 ms
 constexpr int kFwdCols = kTile / kFwdGroups;     // keys per group and tile
-constexpr int kFwdEpiWarps = 4;                    // fast pass: warps that write O and LSE out and stage Q
+constexpr int kFwdEpiWarps = 8;                    // fast pass: warps that write O and LSE out and stage Q
 constexpr int kFwdThreads = 128 * kFwdGroups + 64 + 32 * kFwdEpiWarps;
 constexpr int kFwdBarSlots = 32;                 // mbarriers of one pass
 constexpr int kFwdMaxUnits = 1024;               // work units one CTA may walk (one redo bit each)
@@ -218,9 +218,9 @@ struct FwdFastBars {
   uint64_t *q_full, *k01, *ready, *sdone, *o_full, *o_free, *stats_full;
   __device__ explicit FwdFastBars(uint64_t* b)
       : q_full(b), k01(b + 2), ready(b + 3), sdone(b + 7), o_full(b + 11), o_free(b + 12), stats_full(b + 13) {}
-  __device__ void init() const {
-    mbar_init(q_full, 32 * kFwdEpiWarps);
-    mbar_init(q_full + 1, 32 * kFwdEpiWarps);
+  __device__ void init(int q_count) const {
+    mbar_init(q_full, q_count);
+    mbar_init(q_full + 1, q_count);
     mbar_init(k01, 1);
     for (int i = 0; i < 4; ++i) { mbar_init(ready + i, 1 + 128 * kFwdGroups); mbar_init(sdone + i, 1); }
     mbar_init(o_full, 1);
@@ -685,26 +685,28 @@ __device__ __forceinline__ void fwd_softmax_fast(const FwdUnit<D>& u, const FwdS
 }
 
 // ---------------------------------------------------------------------------------- epilogue warps, fast pass
-// Four warps (one per quarter of the tensor-memory lanes; lane = query row of the tile).  Per unit: wait for the row
-// statistics and for the last P V, read O out of tensor memory (two 32-column slices at a time; o_free after the last
-// read), normalise, store O and LSE; then fetch the Q rows of the unit after the next into the Q buffer this unit used.
+// Eight warps: one per quarter of the tensor-memory lanes (lane = query row of the tile) and half of the head
+// dimension.  Per unit: wait for the row statistics and for the last P V, read the warp's half of O out of tensor
+// memory in one go (o_free right after), normalise, store O (and LSE: the first half's warps); then fetch the warp's
+// 64-element part of the Q rows of the unit after the next into the Q buffer this unit used.
 // They keep every load from and store to global memory away from the softmax threads.
 template <int D>
 __device__ __forceinline__ void fwd_epilogue_fast(const FwdUnit<D>& u, const FwdSched& sch, const FwdFastBars& bar,
                                                   int warp, int lane, const __nv_bfloat16* q, int n_q, int heads,
                                                   __nv_bfloat16* o, float* lse, uint32_t* redo_bits) {
-  constexpr int kSlices = D / 32;
+  constexpr int kSlices = D / 32, kOwn = kSlices / 2;   // 32-column slices of O: all, and this warp's
+  constexpr int kMmaWarp = 4 * kFwdGroups;
   const FwdStats<D> stats{u.smax};
+  const int half = (warp - kMmaWarp - 2) >> 2;          // 0: columns [0, D/2), 1: the others
   const int r = (warp & 3) * 32 + lane;
   const uint32_t tmem_lane = u.tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+  const bool stages_q = half < D / 64;                  // part `half` of the Q rows
   auto stage_q = [&](const FwdPos& pos, int buf) {
+    if (!stages_q) return;
     const FwdRow<D> row(sch, pos, r, q, n_q, heads, o, lse);
-#pragma unroll
-    for (int part = 0; part < D / 64; ++part) {
-      uint32_t qr[32];
-      row.load_q(qr, part, lane);
-      tmem_st32(tmem_lane + kFwdColQ + buf * kFwdQCols + part * 32, qr);
-    }
+    uint32_t qr[32];
+    row.load_q(qr, half, lane);
+    tmem_st32(tmem_lane + kFwdColQ + buf * kFwdQCols + half * 32, qr);
     tmem_wait_st();
     tc_fence_before_sync();
     mbar_arrive(bar.q_full + buf);
@@ -731,20 +733,15 @@ __device__ __forceinline__ void fwd_epilogue_fast(const FwdUnit<D>& u, const Fwd
     uint64_t chk2 = f32x2(0.f, 0.f);
     mbar_wait(bar.o_full, n & 1, u.abort_flag);
     tc_fence_after_sync();
+    uint32_t acc[kOwn][32];
 #pragma unroll
-    for (int c4 = 0; c4 < kSlices; c4 += 2) {
-      uint32_t acc[2][32];
-      tmem_ld32(tmem_lane + kFwdColO + c4 * 32, acc[0]);
-      tmem_ld32(tmem_lane + kFwdColO + (c4 + 1) * 32, acc[1]);
-      tmem_wait_ld();
-      if (c4 + 2 >= kSlices) {   // O is in registers (or stored): the next unit may start on it
-        tc_fence_before_sync();
-        mbar_arrive(bar.o_free);
-      }
-      fwd_store_slice(acc[0], inv2, chk2, row.out, c4 * 32, lane);
-      fwd_store_slice(acc[1], inv2, chk2, row.out, (c4 + 1) * 32, lane);
-    }
-    if (row.in_range && row.lse_dst != nullptr) *row.lse_dst = (m + log2f(l)) * 0.6931471805599453f;
+    for (int i = 0; i < kOwn; ++i) tmem_ld32(tmem_lane + kFwdColO + (half * kOwn + i) * 32, acc[i]);
+    tmem_wait_ld();
+    tc_fence_before_sync();
+    mbar_arrive(bar.o_free);   // this warp's part of O is in registers: the next unit may start on it
+#pragma unroll
+    for (int i = 0; i < kOwn; ++i) fwd_store_slice(acc[i], inv2, chk2, row.out, (half * kOwn + i) * 32, lane);
+    if (half == 0 && row.in_range && row.lse_dst != nullptr) *row.lse_dst = (m + log2f(l)) * 0.6931471805599453f;
     if (!fwd_all_finite(chk2)) atomicOr(redo_bits + (n >> 5), 1u << (n & 31));
     // Q of the unit after the next, into this unit's buffer: every S of this unit is complete (o_full)
     if (unit + 2 * sch.stride < sch.total) {
@@ -918,7 +915,7 @@ chunk_attn_fwd_kernel(const __nv_bfloat16* __restrict__ q, const __grid_constant
     tma_prefetch_desc(&tm_kc); tma_prefetch_desc(&tm_vc); tma_prefetch_desc(&tm_kx); tma_prefetch_desc(&tm_vx0);
   }
   if (tid == 0) {
-    bar_fast.init();
+    bar_fast.init(128 * (D / 64));   // q_full: one arrival per row and 64-element part
     bar_safe.init(1, 128);
     *abort_flag = 0;
     fence_mbar_init();
