@@ -530,3 +530,46 @@ def test_group_of_24_candidates_on_one_shared_prefix(mode):
         kx, vx = orc.bf16_bits_to_f64(mk[:, :, h:h + 1, :]), orc.bf16_bits_to_f64(mv[:, :, h:h + 1, :])
         o_ref, lse_ref = orc.chunk_attn_fwd(sl(bits[0])[:, rows], kx, vx, sl(bits[1]), sl(bits[2]), w.scale)
         check_fwd(o[b:b + 1, rows, h:h + 1], lse[b:b + 1, h:h + 1][:, :, rows], o_ref, lse_ref, tag="b%d h%d" % (b, h))
+
+
+@pytest.mark.parametrize("n_k", [100, 200, 3 * 128, 5 * 128 + 9])
+def test_more_work_units_than_sms_with_few_key_tiles(n_k):
+    """240 (query tile, head, sample) units of 1, 2, 3 or 6 key tiles each: every CTA walks over two of them, so
+    the S look-ahead, the K/V rings and the two Q buffers all cross unit boundaries, with units shorter than the
+    look-ahead itself; the last query tile is ragged."""
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, n_q = 3, 20, 128, 3 * 128 + 16
+    qb = synth.normal_bf16(5101, (B, n_q, H, D)); kb = synth.normal_bf16(5102, (B, n_k, H, D))
+    vb = synth.normal_bf16(5103, (B, n_k, H, D))
+    q, k, v = (dev_bf16(x) for x in (qb, kb, vb))
+    qf, kf, vf = (orc.bf16_bits_to_f64(x) for x in (qb, kb, vb))
+    scale = 1.0 / np.sqrt(D)
+    o, lse = A.astro_chunk_attn_fwd(None, q, k, v, scale)
+    A.astro_last_device_status()
+    o_ref, lse_ref = orc.chunk_attn_fwd(qf, None, None, kf, vf, scale)
+    check_fwd(o, lse, o_ref, lse_ref)
+
+
+def test_some_units_of_a_cta_need_the_safe_pass():
+    """444 units of three key tiles; in heads 1 and 4 the keys of the later tiles are scaled up so far that the rows'
+    sums overflow against their first-tile reference.  Only the units of those heads are redone by the safe pass;
+    they sit between units of other heads in the walk of one CTA."""
+    import torch
+    from paper_2603_17051_b200 import binding as A
+    B, H, D, n_q, n_k = 2, 6, 128, 37 * 128 - 50, 3 * 128
+    qb = synth.normal_bf16(5201, (B, n_q, H, D)); kb = synth.normal_bf16(5202, (B, n_k, H, D))
+    vb = synth.normal_bf16(5203, (B, n_k, H, D))
+    kf = orc.bf16_bits_to_f64(kb)
+    gain = 1.0 + 30.0 * (np.arange(n_k) // 128)
+    for h in (1, 4):
+        kf[:, :, h] *= gain[None, :, None]
+    kb = synth.f32_to_bf16_bits(kf.astype(np.float32))
+    q, k, v = (dev_bf16(x) for x in (qb, kb, vb))
+    qf, kf, vf = (orc.bf16_bits_to_f64(x) for x in (qb, kb, vb))
+    scale = 1.0 / np.sqrt(D)
+    o, lse = A.astro_chunk_attn_fwd(None, q, k, v, scale)
+    A.astro_last_device_status()
+    rows = np.concatenate([np.arange(0, n_q, 97), np.arange(n_q - 40, n_q)])   # sampled rows and the ragged tile
+    o_ref, lse_ref = orc.chunk_attn_fwd(qf[:, rows], None, None, kf, vf, scale)
+    pick = torch.from_numpy(rows).to(o.device)
+    check_fwd(o[:, pick], lse[:, :, pick], o_ref, lse_ref, sharp=True)
