@@ -218,11 +218,16 @@ chunk_attn_bwd_dq_kernel(const __nv_bfloat16* __restrict__ q, const __grid_const
     // Q row -> tensor memory: group g writes elements [64g, 64g+64) of its row as 32 packed columns
     if (g * 64 < D) {
       uint32_t qr[32];
-      const uint4* src = reinterpret_cast<const uint4*>(q + ((static_cast<size_t>(b) * n_q + (in_range ? row : 0)) * heads + h) * D + g * 64);
+      const QuadRows q_rows = quad_rows(q, b, h, n_q, heads, D, row);   // the quads of a warp fetch their rows together
 #pragma unroll
-      for (int v = 0; v < 8; ++v) {
-        const uint4 t = in_range ? src[v] : make_uint4(0, 0, 0, 0);
-        qr[4 * v] = t.x; qr[4 * v + 1] = t.y; qr[4 * v + 2] = t.z; qr[4 * v + 3] = t.w;
+      for (int half = 0; half < 2; ++half) {
+        uint4 ch[4];
+        load_quad_rows(ch, q_rows, g * 64 + half * 32, tid & 31);
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          qr[16 * half + 4 * v] = ch[v].x; qr[16 * half + 4 * v + 1] = ch[v].y;
+          qr[16 * half + 4 * v + 2] = ch[v].z; qr[16 * half + 4 * v + 3] = ch[v].w;
+        }
       }
       tmem_st32(tmem_lane + kColQ + g * 32, qr);
       tmem_wait_st();

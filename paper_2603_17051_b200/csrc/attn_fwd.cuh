@@ -1,11 +1,12 @@
-// Forward of chunk attention over the rolling cache: O and LSE for one 128-query tile per CTA.
+// Forward of chunk attention over the rolling cache: O and LSE.  A work unit is one 128-query tile of one head of
+// one sample; one CTA per SM walks over its share of the units.
 //
-// Warp-specialised, one CTA per SM:
+// Warp-specialised:
 //   four softmax groups of 4 warps: group g owns keys [32 g, 32 g + 32) of every key tile, one query row
 //   per thread (four warps per scheduler: while one waits for tensor memory or a barrier the others keep the
 //   special-function unit busy); then one warp whose first thread issues every tcgen05 MMA, one for TMA loads, and
-//   eight epilogue warps that write O and LSE out and bring the next units' Q rows in (fast pass)
-// Q lives in tensor memory (bf16 pairs, written once by the softmax threads) and is the A operand of
+//   (fast pass) eight epilogue warps that write O and LSE out and bring the Q rows of the units to come in.
+// Q lives in tensor memory (bf16 pairs, two buffers: the unit at hand and the next) and is the A operand of
 // S = Q K^T, so shared memory only carries K and V: an MMA with both operands in shared memory reads
 // 128 B/clk, the whole shared-memory bandwidth, and then competes with the TMA writes of the next tiles.
 // S of a whole key tile is one 128x128 MMA into one of two S buffers, issued two tiles ahead.  P is written
@@ -14,17 +15,20 @@
 // the special-function unit (16 exp2 per clock per SM, as busy as the tensor core at head_dim 128); measured, the
 // polynomial's own FMA and integer work costs more than it saves, so the share is zero.
 //
-// The kernel makes up to two passes over the keys:
-//   fast pass  every row keeps ONE reference exponent, the maximum of its first key tile.  exp2(s - m) is
-//              exact for any reference as long as nothing overflows (bf16 and fp32 share the exponent range,
-//              so later scores may exceed the reference by ~100 in log2 units), so O is never rescaled, the
-//              threads of a row never have to agree on anything after the first tile.  The MMA-issuing thread
-//              sets the pace, so everything a tile needs (the bytes of V(j) and K(j+2), every thread's P(j))
-//              arrives on ONE barrier and every burst of 16 MMAs (P V of tile j, S of tile j+2) is followed by
-//              ONE commit.
-//   safe pass  only if some row of the CTA saw a sum beyond 2^100, an infinity or a NaN in the fast pass: the
-//              whole tile is recomputed with a running reference that follows the row maximum (rescaling O
-//              and the row sums when a tile's row sum leaves the safe range).
+// The kernel makes up to two passes:
+//   fast pass  over all the CTA's units.  Every row keeps ONE reference exponent, the maximum of its first key
+//              tile.  exp2(s - m) is exact for any reference as long as nothing overflows (bf16 and fp32 share the
+//              exponent range, so later scores may exceed the reference by ~100 in log2 units), so O is never
+//              rescaled and the threads of a row never have to agree on anything after the first tile.  The
+//              MMA-issuing thread sets the pace, so everything a tile needs (the bytes of V(J) and K(J+2), every
+//              thread's P(J)) arrives on ONE barrier and every burst of 16 MMAs (P V of tile J, S of tile J+2) is
+//              followed by ONE commit.  The key tiles of all the CTA's units form one stream: look-ahead, rings
+//              and barriers run on across unit boundaries, where the softmax threads only leave their row sums
+//              and references in shared memory; the epilogue warps do everything else there (O out of tensor
+//              memory, normalised, stored; LSE; the Q rows of the unit after the next into the free Q buffer).
+//   safe pass  unit by unit, only for units one of whose rows saw a sum beyond 2^100, an infinity or a NaN in the
+//              fast pass: the unit is recomputed with a running reference that follows the row maximum (rescaling
+//              O and the row sums when a tile's row sum leaves the safe range).
 //   TMEM columns: S buffers [0,128) [128,256)   O [256,256+D)   Q buffers [384,384+D/2) [448,448+D/2)
 #pragma once
 #include <type_traits>
@@ -36,7 +40,7 @@ namespace astro {
 constexpr int kFwdKStages = 3, kFwdVStages = 3, kFwdSBufs = 2;
 constexpr int kFwdGroups = 4;                    // layer shape, forward alone: 2 groups 0.741 ms, 4 groups 0.713 ms
 constexpr int kFwdCols = kTile / kFwdGroups;     // keys per group and tile
-constexpr int kFwdEpiWarps = 8;                    // fast pass: warps that write O and LSE out and stage Q
+constexpr int kFwdEpiWarps = 8;                  // fast pass: warps that write O and LSE out and stage Q
 constexpr int kFwdThreads = 128 * kFwdGroups + 64 + 32 * kFwdEpiWarps;
 constexpr int kFwdBarSlots = 32;                 // mbarriers of one pass
 constexpr int kFwdMaxUnits = 1024;               // work units one CTA may walk (one redo bit each)
@@ -53,7 +57,7 @@ template <int D> struct FwdSmem {
 // 0 -> 0.776 ms, 1 -> 0.781, 2 -> 0.802, 3 -> 0.828 in bursts; the same order under the power limit.
 constexpr int kPolyOf8 = 0;
 constexpr float kRowSumLimit = 1073741824.f;        // safe pass: a tile row sum beyond 2^30 re-references the row
-constexpr float kFastSumLimit = 1.2676506e30f;      // fast pass: a row sum beyond 2^100 sends the CTA to the safe pass
+constexpr float kFastSumLimit = 1.2676506e30f;      // fast pass: a row sum beyond 2^100 sends the unit to the safe pass
 constexpr float kPolyArgLimit = 126.f;              // largest exponent the polynomial exp2 may be handed
 
 // The mbarriers of the safe pass.  The two passes use separate sets, so a late arrival of the first pass can
