@@ -54,7 +54,8 @@ template <int D> struct FwdSmem {
 };
 
 // Of every 8 pairs of exponentials, how many use the polynomial on the FMA pipe.  Layer shape, forward alone:
-// 0 -> 0.776 ms, 1 -> 0.781, 2 -> 0.802, 3 -> 0.828 in bursts; the same order under the power limit.
+// 0 -> 0.776 ms, 1 -> 0.781, 2 -> 0.802, 3 -> 0.828 in bursts; the same order under the power limit.  The same
+// again with four softmax groups and the CTAs walking over their units: 0 -> 0.662 ms, 1 -> 0.689, 2 -> 0.719.
 constexpr int kPolyOf8 = 0;
 constexpr float kRowSumLimit = 1073741824.f;        // safe pass: a tile row sum beyond 2^30 re-references the row
 constexpr float kFastSumLimit = 1.2676506e30f;      // fast pass: a row sum beyond 2^100 sends the unit to the safe pass
@@ -610,7 +611,6 @@ __device__ __forceinline__ void fwd_fast_tile(const FwdTileCtx& c, int J, int va
 // Returns the row sum.
 __device__ __noinline__ float fwd_fast_run(uint32_t tmem_lane_g, uint32_t sdone, uint32_t ready, uint32_t abort_flag,
                                            float scale_log2, float neg_m, float l_run, int J, int count) {
-  static_assert(kPolyOf8 == 0, "the out-of-line loop leaves the polynomial's range check out");
   static_assert(kFwdCols == 32, "one 32-column load per thread and tile");
   float poly_max = -INFINITY;
   for (int i = 0; i < count; ++i, ++J) {
@@ -626,6 +626,7 @@ __device__ __noinline__ float fwd_fast_run(uint32_t tmem_lane_g, uint32_t sdone,
     tc_fence_before_sync();
     mbar_arrive_at(ready + 8 * (J % 4));
   }
+  if (poly_max > kPolyArgLimit) l_run = INFINITY;   // the polynomial was handed an argument beyond its range: redo the unit
   return l_run;
 }
 
