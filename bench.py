@@ -413,16 +413,22 @@ def run_ours(args):
     dom = max(kernel_flops, key=lambda k: stage_ms[k])
     kname, kflops = kernel_flops[dom]
     achieved = kflops / (stage_ms[dom] * 1e-3) / 1e12
-    # A timed region of under a second runs at burst clocks, a longer one settles at the board's power limit:
-    # compare with the cuBLAS figure measured in the same regime, and give the other fraction beside it.
+    # A short timed region runs at burst clocks, a longer one settles at the board's power limit: compare with the
+    # cuBLAS figure measured in the same regime, and give the other fraction beside it.  The regime is read off the
+    # clocks sampled during the region (power cap active and the median SM clock under 90 % of its maximum: the
+    # region ran power-capped, however short it was); without samples, off its length.
     timed_s = (t_wall1 - t_wall0)
-    regime = "burst" if timed_s < 1.0 else "sustained"
+    capped = ("sw_power_cap" in (clocks.get("reasons") or [])) and \
+        (clocks.get("sm_mhz") or 0) < 0.9 * (clocks.get("sm_max_mhz") or 1e9)
+    regime = "sustained" if (timed_s >= 1.0 or capped) else "burst"
     peak = peaks["bf16_" + regime]
     traffic = ncu_traffic()
     roofline = {"bound": "tensor", "kernel": kname, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak, "traffic": traffic[dom], "traffic_unit": "bytes of DRAM traffic per launch",
-                "peak_source": "%s cuBLAS bf16 %s figure (timed region %.2f s); burst %.1f, sustained %.1f" % (
-                    peaks["source"], regime, timed_s, peaks["bf16_burst"], peaks["bf16_sustained"]),
+                "peak_source": "%s cuBLAS bf16 %s figure (timed region %.2f s, SM clock median %s MHz%s); burst %.1f, "
+                               "sustained %.1f" % (peaks["source"], regime, timed_s, clocks.get("sm_mhz"),
+                                                   ", power cap active" if capped else "", peaks["bf16_burst"],
+                                                   peaks["bf16_sustained"]),
                 "frac_of_burst": achieved / peaks["bf16_burst"], "frac_of_sustained": achieved / peaks["bf16_sustained"],
                 "frac_of_nominal_2250": achieved / 2250.0, "ms_per_launch": stage_ms[dom],
                 "algorithmic_flops_per_launch": kflops}
